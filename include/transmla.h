@@ -1,0 +1,186 @@
+/*
+ * transmla.h - C ABI of the absorbed-MLA decode library for NVIDIA B200 (sm_100a).
+ *
+ * The library computes one attention layer's decode step for a GQA model converted to
+ * Multi-head Latent Attention (TransMLA, arXiv 2502.07864), in the Absorb form (Sec. 3.3, Eq. 9
+ * right-hand column) directly over the compressed per-token latent cache
+ *     k_hat_t = [ c_t^KV ; k_t^R ]        (r + dR values per token and layer).
+ *
+ * Symbols follow the paper: D hidden size, H (= h) query heads, dn (= d) per-head no-RoPE key dim,
+ * dR (= d^R) decoupled RoPE dim, dv per-head value dim, r (= r_kv) latent rank; B sequences,
+ * S new query tokens per sequence, L_b cached tokens of sequence b (the S new ones included),
+ * P tokens per cache page.
+ *
+ * General rules for every entry point
+ *   - "device" pointers are CUDA device memory of the current device, "host" pointers are ordinary
+ *     host memory.  The caller owns every buffer.  Unless an entry point says otherwise the library
+ *     allocates nothing, frees nothing, never synchronises, and enqueues work only on `stream`
+ *     (a cudaStream_t passed as void*; NULL = the default stream).
+ *   - All floating-point tensors are bfloat16 unless stated, dense, row-major, last index fastest.
+ *     Accumulation is fp32; casts to bf16 round to nearest even.
+ *   - Tensor bases must be 16-byte aligned; the cache base 128-byte aligned.
+ *   - Problems that the host can see (null or misaligned pointer, unsupported shape, workspace too
+ *     small, no sm_100 device) return an error code and launch nothing.  Problems only the device can
+ *     see set bits in `*dev_status` (device int32, may be NULL; the caller zeroes it and reads it
+ *     after synchronising) and never trap: a page-table entry outside [0, num_pages) is skipped
+ *     (its tokens contribute nothing) and sets TRANSMLA_DEV_BAD_PAGE; a bounded wait that expired
+ *     sets TRANSMLA_DEV_TIMEOUT and the affected results are unspecified.
+ *   - Thread safety: no global mutable state except a cache of TMA descriptors guarded by a mutex.
+ */
+#ifndef TRANSMLA_H_
+#define TRANSMLA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  TRANSMLA_OK = 0,
+  TRANSMLA_ERR_NULL = 1,      /* a required pointer is NULL */
+  TRANSMLA_ERR_ALIGN = 2,     /* a pointer violates the alignment rule */
+  TRANSMLA_ERR_SHAPE = 3,     /* unsupported or inconsistent dimensions */
+  TRANSMLA_ERR_RANGE = 4,     /* a sequence length or page index is out of range (host validation) */
+  TRANSMLA_ERR_WORKSPACE = 5, /* workspace or staging buffer too small */
+  TRANSMLA_ERR_CUDA = 6,      /* a CUDA runtime/driver call failed */
+  TRANSMLA_ERR_ARCH = 7       /* the current device is not compute capability 10.x */
+} transmla_status_t;
+
+/* bits of the device status word */
+#define TRANSMLA_DEV_BAD_PAGE 1
+#define TRANSMLA_DEV_TIMEOUT 2
+
+typedef struct {
+  int32_t hidden_dim;        /* D; used by the append only */
+  int32_t num_heads;         /* H */
+  int32_t q_len;             /* S >= 1 */
+  int32_t qk_nope_dim;       /* dn */
+  int32_t qk_rope_dim;       /* dR, even, may be 0 */
+  int32_t v_dim;             /* dv */
+  int32_t kv_lora_rank;      /* r */
+  int32_t page_size;         /* P; must be 64 */
+  int32_t num_pages;         /* pages in the cache pool */
+  int32_t max_pages_per_seq; /* row stride of page_table */
+  int32_t batch;             /* B */
+  int32_t num_partitions;    /* G: how many pieces the batch's pages are split into; 0 = library chooses */
+  float softmax_scale;       /* 1/sqrt(dn + dR) for MLA (Eq. 9), 1/sqrt(d) for a lifted GQA layer (Eq. 13) */
+  float rope_theta;          /* RoPE base, 10000 in Eq. 1 */
+} transmla_params_t;
+
+/* Supported (r, dR) pairs: (512, 64), (128, 0), (64, 16).  dn, dv: multiples of 8 up to 256.
+ * S*H <= 1024.  page_size == 64. */
+
+/* Byte offsets of the regions inside the workspace that carries results from
+ * transmla_mla_decode to transmla_mla_combine.  All regions are written by transmla_mla_decode.
+ *   q_hat       bf16  [B, S, H, r+dR]   absorbed queries (Eq. 9 right, first line)
+ *   cum_pages   int32 [B+1]             cum[b] = sum_{b'<b} ceil(L_b'/P)
+ *   plan        int32 [G, 4]            per partition: flat page begin, end, sequence of first page,
+ *                                       sequence of last page (-1, -1 for an empty partition);
+ *                                       partition i owns flat pages [floor(i*T/G), floor((i+1)*T/G)),
+ *                                       T = cum[B]
+ *   partial_o   fp32  [G+B-1, S*H, r]   per segment (partition i, sequence b), slot = i + b:
+ *                                       softmax-weighted mean of c_j over the segment's visible tokens
+ *   partial_lse fp32  [G+B-1, S*H]      natural-log softmax denominator of the segment (-inf = empty)
+ * Row index inside a slot is s*H + h. */
+typedef struct {
+  int32_t num_partitions;  /* the G actually used */
+  int32_t num_slots;       /* G + B - 1 */
+  size_t q_hat_offset;
+  size_t cum_pages_offset;
+  size_t plan_offset;
+  size_t partial_o_offset;
+  size_t partial_lse_offset;
+  size_t total_bytes;
+} transmla_workspace_layout_t;
+
+/* Workspace layout and size for `params` (host computation only; needs a CUDA device only when
+ * params->num_partitions == 0, to read its SM count).  Returns TRANSMLA_OK or an error. */
+transmla_status_t transmla_workspace_layout(const transmla_params_t* params /* host */,
+                                            transmla_workspace_layout_t* layout /* host, out */);
+
+/* Latent append (Sec. 3.3, Eq. 7 left column):
+ *     c_t = W_DKV x_t,   k_t^R = RoPE(W_KR x_t, t)   (RoPE of Eq. 1: interleaved pairs, angle
+ *     t * rope_theta^(-2l/dR) for pair l), rounded to bf16 and stored as the cache row of token t.
+ * Token (b, s) has position positions[b] + s and goes to
+ *     cache[page_table[b][pos / P]][pos % P][0 .. r+dR).
+ *   x          device bf16 [B, S, D]
+ *   w_dkv_kr   device bf16 [r+dR, D]: rows 0..r-1 = W_DKV, rows r.. = W_KR
+ *   positions  device int32 [B], 0-based position of each sequence's first new token
+ *   page_table device int32 [B, max_pages_per_seq]
+ *   cache      device bf16 [num_pages, P, r+dR]; only the addressed rows are written
+ * A position that maps outside the page table or to a page outside the pool is skipped and sets
+ * TRANSMLA_DEV_BAD_PAGE. */
+transmla_status_t transmla_latent_append(const transmla_params_t* params /* host */,
+                                         const void* x, const void* w_dkv_kr, const int32_t* positions,
+                                         const int32_t* page_table, void* cache, int32_t* dev_status,
+                                         void* stream);
+
+/* Absorb + split-KV decode (Eq. 9 right column, first and second line):
+ *     q_hat[b,s,h] = [ W_UK_h^T q_nope[b,s,h] ; q_pe[b,s,h] ]
+ *     o_hat[b,s,h] = sum_j softmax_j( q_hat . k_hat_j * softmax_scale ) c_j
+ * over the visible tokens j in [0, L_b - (S-1-s)) of sequence b (the cache already holds the S new
+ * tokens; query s sees everything up to and including its own token).  The batch's pages are split
+ * into G partitions (see transmla_workspace_layout_t); each segment's normalised partial result and
+ * log-sum-exp go to the workspace.  Rows of a page beyond L_b, and page-table entries beyond
+ * ceil(L_b/P), are never used and may hold anything (NaN included).
+ *   q_nope     device bf16 [B, S, H, dn]
+ *   q_pe       device bf16 [B, S, H, dR]  RoPE already applied (ignored when dR == 0; may be NULL then)
+ *   w_uk       device bf16 [H, dn, r]     k^C_h = W_UK_h c
+ *   cache      device bf16 [num_pages, P, r+dR]
+ *   page_table device int32 [B, max_pages_per_seq]
+ *   seqlens    device int32 [B], 0 <= L_b <= max_pages_per_seq * P
+ *   workspace  device, >= layout.total_bytes, 256-byte aligned */
+transmla_status_t transmla_mla_decode(const transmla_params_t* params /* host */, const void* q_nope,
+                                      const void* q_pe, const void* w_uk, const void* cache,
+                                      const int32_t* page_table, const int32_t* seqlens, void* workspace,
+                                      size_t workspace_bytes, int32_t* dev_status, void* stream);
+
+/* Combine + up-projection (Eq. 9 right column, last line, before W_O):
+ *     o_hat = sum_k w_k partial_o_k,  w_k = exp(lse_k - lse) with lse = log sum_k exp(lse_k),
+ *     out[b,s,h] = W_UV_h o_hat[b,s,h].
+ * Reads cum_pages, partial_o and partial_lse from the workspace a preceding transmla_mla_decode
+ * with the same `params` filled.
+ *   w_uv       device bf16 [H, dv, r]     v_h = W_UV_h c
+ *   out        device bf16 [B, S, H, dv]
+ *   lse_out    device fp32 [B, S, H] or NULL; natural log of the full softmax denominator
+ * A query that sees no token (L_b - (S-1-s) <= 0) gets out = 0 and lse = -inf. */
+transmla_status_t transmla_mla_combine(const transmla_params_t* params /* host */, const void* workspace,
+                                       size_t workspace_bytes, const void* w_uv, void* out,
+                                       float* lse_out, int32_t* dev_status, void* stream);
+
+/* Host-side check of the index tables (host pointers): every L_b in [0, max_pages_per_seq*P], every
+ * used page-table entry in [0, num_pages), no page used twice.  Returns TRANSMLA_OK or
+ * TRANSMLA_ERR_RANGE.  Launches nothing. */
+transmla_status_t transmla_validate_tables(const transmla_params_t* params /* host */,
+                                           const int32_t* page_table /* host */,
+                                           const int32_t* seqlens /* host */);
+
+/* Bytes of device staging transmla_decode_step_host needs for `params`. */
+size_t transmla_step_staging_bytes(const transmla_params_t* params /* host */);
+
+/* One whole decode step driven from host buffers: validates the tables, copies this step's inputs to
+ * the device (x, q_nope, q_pe, page_table, seqlens), appends the S new tokens of every sequence at
+ * positions L_b - S .. L_b - 1, runs decode and combine, copies `out` (and `lse` if not NULL) back
+ * and waits for `stream`.  Weights and the cache stay resident on the device.  Host buffers should
+ * be pinned for the copies to be asynchronous.  Returns the first error, or TRANSMLA_OK;
+ * `*h_dev_status` (host, may be NULL) receives the device status word.
+ *   h_x [B,S,D], h_q_nope [B,S,H,dn], h_q_pe [B,S,H,dR], h_page_table, h_seqlens : host
+ *   w_dkv_kr, w_uk, w_uv, cache, staging, workspace                              : device
+ *   h_out [B,S,H,dv] bf16, h_lse [B,S,H] fp32 or NULL                            : host */
+transmla_status_t transmla_decode_step_host(const transmla_params_t* params, const void* h_x,
+                                            const void* h_q_nope, const void* h_q_pe,
+                                            const int32_t* h_page_table, const int32_t* h_seqlens,
+                                            const void* w_dkv_kr, const void* w_uk, const void* w_uv,
+                                            void* cache, void* staging, size_t staging_bytes,
+                                            void* workspace, size_t workspace_bytes, void* h_out,
+                                            float* h_lse, int32_t* h_dev_status, void* stream);
+
+/* Human-readable name of a status code (static storage). */
+const char* transmla_status_string(transmla_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TRANSMLA_H_ */

@@ -1,0 +1,166 @@
+"""ctypes binding of libtransmla.so: argument marshalling only, same names as the C ABI.
+
+Every computation runs in the library's CUDA kernels.  There is no CPU fallback: if the library
+is missing or was not built, importing a function from here raises.
+"""
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, 'libtransmla.so')
+
+EXPORTS = ('transmla_workspace_layout', 'transmla_latent_append', 'transmla_mla_decode', 'transmla_mla_combine',
+           'transmla_validate_tables', 'transmla_step_staging_bytes', 'transmla_decode_step_host',
+           'transmla_status_string')
+
+
+class Params(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        'hidden_dim', 'num_heads', 'q_len', 'qk_nope_dim', 'qk_rope_dim', 'v_dim', 'kv_lora_rank', 'page_size',
+        'num_pages', 'max_pages_per_seq', 'batch', 'num_partitions')] + [
+        ('softmax_scale', ctypes.c_float), ('rope_theta', ctypes.c_float)]
+
+
+class WorkspaceLayout(ctypes.Structure):
+    _fields_ = [('num_partitions', ctypes.c_int32), ('num_slots', ctypes.c_int32),
+                ('q_hat_offset', ctypes.c_size_t), ('cum_pages_offset', ctypes.c_size_t),
+                ('plan_offset', ctypes.c_size_t), ('partial_o_offset', ctypes.c_size_t),
+                ('partial_lse_offset', ctypes.c_size_t), ('total_bytes', ctypes.c_size_t)]
+
+
+class TransMLAError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        super().__init__(f'{where}: {status_string(code)} (status {code})')
+
+
+_lib = None
+
+
+def lib():
+    """The loaded library; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError(f'{_LIB_PATH} is missing: build it with `python -m paper_2502_07864_b200.build`')
+        L = ctypes.CDLL(_LIB_PATH)
+        vp, i32p, sz = ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t
+        pp = ctypes.POINTER(Params)
+        L.transmla_workspace_layout.argtypes = [pp, ctypes.POINTER(WorkspaceLayout)]
+        L.transmla_latent_append.argtypes = [pp, vp, vp, i32p, i32p, vp, i32p, vp]
+        L.transmla_mla_decode.argtypes = [pp, vp, vp, vp, vp, i32p, i32p, vp, sz, i32p, vp]
+        L.transmla_mla_combine.argtypes = [pp, vp, sz, vp, vp, vp, i32p, vp]
+        L.transmla_validate_tables.argtypes = [pp, i32p, i32p]
+        L.transmla_step_staging_bytes.argtypes = [pp]
+        L.transmla_step_staging_bytes.restype = sz
+        L.transmla_decode_step_host.argtypes = [pp, vp, vp, vp, i32p, i32p, vp, vp, vp, vp, vp, sz, vp, sz, vp, vp,
+                                                i32p, vp]
+        L.transmla_status_string.argtypes = [ctypes.c_int]
+        L.transmla_status_string.restype = ctypes.c_char_p
+        for name in EXPORTS:
+            if name not in ('transmla_step_staging_bytes', 'transmla_status_string'):
+                getattr(L, name).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def status_string(code):
+    return lib().transmla_status_string(int(code)).decode()
+
+
+def make_params(shape, batch, num_pages, max_pages_per_seq, softmax_scale, num_partitions=0, rope_theta=10000.0):
+    """Params from an MLAShape-like object (attributes H, S, dn, dR, dv, r, D, page_size)."""
+    return Params(hidden_dim=shape.D, num_heads=shape.H, q_len=shape.S, qk_nope_dim=shape.dn,
+                  qk_rope_dim=shape.dR, v_dim=shape.dv, kv_lora_rank=shape.r, page_size=shape.page_size,
+                  num_pages=num_pages, max_pages_per_seq=max_pages_per_seq, batch=batch,
+                  num_partitions=num_partitions, softmax_scale=softmax_scale, rope_theta=rope_theta)
+
+
+def _ptr(t):
+    return ctypes.c_void_p(0 if t is None else t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _check(code, where):
+    if code != 0:
+        raise TransMLAError(code, where)
+
+
+def transmla_workspace_layout(params):
+    lay = WorkspaceLayout()
+    _check(lib().transmla_workspace_layout(ctypes.byref(params), ctypes.byref(lay)), 'transmla_workspace_layout')
+    return lay
+
+
+def transmla_latent_append(params, x, w_dkv_kr, positions, page_table, cache, dev_status=None, stream=None):
+    _check(lib().transmla_latent_append(ctypes.byref(params), _ptr(x), _ptr(w_dkv_kr), _ptr(positions),
+                                        _ptr(page_table), _ptr(cache), _ptr(dev_status), _stream(stream)),
+           'transmla_latent_append')
+
+
+def transmla_mla_decode(params, q_nope, q_pe, w_uk, cache, page_table, seqlens, workspace, dev_status=None,
+                        stream=None):
+    _check(lib().transmla_mla_decode(ctypes.byref(params), _ptr(q_nope), _ptr(q_pe), _ptr(w_uk), _ptr(cache),
+                                     _ptr(page_table), _ptr(seqlens), _ptr(workspace),
+                                     workspace.numel() * workspace.element_size(), _ptr(dev_status), _stream(stream)),
+           'transmla_mla_decode')
+
+
+def transmla_mla_combine(params, workspace, w_uv, out, lse_out=None, dev_status=None, stream=None):
+    _check(lib().transmla_mla_combine(ctypes.byref(params), _ptr(workspace),
+                                      workspace.numel() * workspace.element_size(), _ptr(w_uv), _ptr(out),
+                                      _ptr(lse_out), _ptr(dev_status), _stream(stream)),
+           'transmla_mla_combine')
+
+
+def transmla_validate_tables(params, page_table_host, seqlens_host):
+    """Host tensors (int32, contiguous).  Returns the status code instead of raising."""
+    return lib().transmla_validate_tables(ctypes.byref(params), _ptr(page_table_host), _ptr(seqlens_host))
+
+
+def transmla_step_staging_bytes(params):
+    return lib().transmla_step_staging_bytes(ctypes.byref(params))
+
+
+def transmla_decode_step_host(params, h_x, h_q_nope, h_q_pe, h_page_table, h_seqlens, w_dkv_kr, w_uk, w_uv, cache,
+                              staging, workspace, h_out, h_lse=None, stream=None):
+    """Returns the device status word."""
+    word = ctypes.c_int32(0)
+    _check(lib().transmla_decode_step_host(
+        ctypes.byref(params), _ptr(h_x), _ptr(h_q_nope), _ptr(h_q_pe), _ptr(h_page_table), _ptr(h_seqlens),
+        _ptr(w_dkv_kr), _ptr(w_uk), _ptr(w_uv), _ptr(cache), _ptr(staging),
+        staging.numel() * staging.element_size(), _ptr(workspace), workspace.numel() * workspace.element_size(),
+        _ptr(h_out), _ptr(h_lse), ctypes.cast(ctypes.byref(word), ctypes.c_void_p), _stream(stream)),
+        'transmla_decode_step_host')
+    return word.value
+
+
+# -------- conveniences built only from the calls above (device-memory plumbing, no arithmetic)
+def alloc_workspace(params, device='cuda'):
+    lay = transmla_workspace_layout(params)
+    return torch.empty(lay.total_bytes, dtype=torch.uint8, device=device), lay
+
+
+def workspace_views(params, workspace, lay=None):
+    """Typed views of the workspace regions (see transmla_workspace_layout_t)."""
+    lay = lay or transmla_workspace_layout(params)
+    B, SH = params.batch, params.q_len * params.num_heads
+    K, r = params.kv_lora_rank + params.qk_rope_dim, params.kv_lora_rank
+
+    def view(off, n, dtype):
+        esz = torch.empty((), dtype=dtype).element_size()
+        return workspace[off:off + n * esz].view(dtype)
+    return {
+        'q_hat': view(lay.q_hat_offset, B * SH * K, torch.bfloat16).view(B, params.q_len, params.num_heads, K),
+        'cum_pages': view(lay.cum_pages_offset, B + 1, torch.int32),
+        'plan': view(lay.plan_offset, lay.num_partitions * 4, torch.int32).view(lay.num_partitions, 4),
+        'partial_o': view(lay.partial_o_offset, lay.num_slots * SH * r, torch.float32).view(lay.num_slots, SH, r),
+        'partial_lse': view(lay.partial_lse_offset, lay.num_slots * SH, torch.float32).view(lay.num_slots, SH),
+    }

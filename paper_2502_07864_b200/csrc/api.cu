@@ -1,0 +1,263 @@
+// C ABI of the absorbed-MLA decode library: argument checks, workspace layout, launches.
+#include <cstdio>
+#include <cstring>
+#include <unordered_set>
+#include <vector>
+
+#include "common.cuh"
+
+using namespace transmla;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+bool supported_latent(int r, int dR) {
+  return (r == 512 && dR == 64) || (r == 128 && dR == 0) || (r == 64 && dR == 16);
+}
+
+transmla_status_t check_shape(const transmla_params_t* p, bool need_hidden) {
+  if (p == nullptr) return TRANSMLA_ERR_NULL;
+  if (p->page_size != kPage) return TRANSMLA_ERR_SHAPE;
+  if (!supported_latent(p->kv_lora_rank, p->qk_rope_dim)) return TRANSMLA_ERR_SHAPE;
+  if (p->num_heads < 1 || p->q_len < 1 || p->num_heads * p->q_len > 1024) return TRANSMLA_ERR_SHAPE;
+  if (p->qk_nope_dim < 8 || p->qk_nope_dim > 256 || p->qk_nope_dim % 8) return TRANSMLA_ERR_SHAPE;
+  if (p->v_dim < 8 || p->v_dim > 256 || p->v_dim % 8) return TRANSMLA_ERR_SHAPE;
+  if (p->batch < 1 || p->num_pages < 1 || p->max_pages_per_seq < 1) return TRANSMLA_ERR_SHAPE;
+  if (p->num_partitions < 0 || p->num_partitions > (1 << 20)) return TRANSMLA_ERR_SHAPE;
+  if (need_hidden && (p->hidden_dim < 8 || p->hidden_dim % 8 || p->hidden_dim > 13312)) return TRANSMLA_ERR_SHAPE;
+  return TRANSMLA_OK;
+}
+
+transmla_status_t check_device(int* sm_count) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return TRANSMLA_ERR_CUDA; }
+  int major = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return TRANSMLA_ERR_CUDA;
+  if (major != 10) return TRANSMLA_ERR_ARCH;
+  if (sm_count != nullptr &&
+      cudaDeviceGetAttribute(sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return TRANSMLA_ERR_CUDA;
+  return TRANSMLA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+transmla_status_t transmla_workspace_layout(const transmla_params_t* p, transmla_workspace_layout_t* out) {
+  if (out == nullptr) return TRANSMLA_ERR_NULL;
+  transmla_status_t st = check_shape(p, false);
+  if (st != TRANSMLA_OK) return st;
+  int G = p->num_partitions;
+  if (G == 0) {
+    int sms = 0;
+    st = check_device(&sms);
+    if (st != TRANSMLA_OK) return st;
+    const int row_blocks = (p->q_len * p->num_heads + kRowBlock - 1) / kRowBlock;
+    G = sms / row_blocks;
+    if (G < 1) G = 1;
+  }
+  const size_t B = p->batch, SH = static_cast<size_t>(p->q_len) * p->num_heads;
+  const size_t K = p->kv_lora_rank + p->qk_rope_dim;
+  const size_t slots = static_cast<size_t>(G) + B - 1;
+  size_t off = 0;
+  out->num_partitions = G;
+  out->num_slots = static_cast<int32_t>(slots);
+  out->q_hat_offset = off;       off = round_up(off + B * SH * K * sizeof(__nv_bfloat16), kAlign);
+  out->cum_pages_offset = off;   off = round_up(off + (B + 1) * sizeof(int32_t), kAlign);
+  out->plan_offset = off;        off = round_up(off + static_cast<size_t>(G) * 4 * sizeof(int32_t), kAlign);
+  out->partial_o_offset = off;   off = round_up(off + slots * SH * p->kv_lora_rank * sizeof(float), kAlign);
+  out->partial_lse_offset = off; off = round_up(off + slots * SH * sizeof(float), kAlign);
+  out->total_bytes = off;
+  return TRANSMLA_OK;
+}
+
+transmla_status_t transmla_latent_append(const transmla_params_t* p, const void* x, const void* w_dkv_kr,
+                                         const int32_t* positions, const int32_t* page_table, void* cache,
+                                         int32_t* dev_status, void* stream) {
+  transmla_status_t st = check_shape(p, true);
+  if (st != TRANSMLA_OK) return st;
+  if (!x || !w_dkv_kr || !positions || !page_table || !cache) return TRANSMLA_ERR_NULL;
+  if (!aligned(x, 16) || !aligned(w_dkv_kr, 16) || !aligned(positions, 4) || !aligned(page_table, 4) ||
+      !aligned(cache, 128) || !aligned(dev_status, 4))
+    return TRANSMLA_ERR_ALIGN;
+  st = check_device(nullptr);
+  if (st != TRANSMLA_OK) return st;
+  cudaError_t e = launch_append(*p, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w_dkv_kr),
+                                positions, page_table, static_cast<__nv_bfloat16*>(cache), dev_status,
+                                static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? TRANSMLA_OK : TRANSMLA_ERR_CUDA;
+}
+
+transmla_status_t transmla_mla_decode(const transmla_params_t* p, const void* q_nope, const void* q_pe,
+                                      const void* w_uk, const void* cache, const int32_t* page_table,
+                                      const int32_t* seqlens, void* workspace, size_t workspace_bytes,
+                                      int32_t* dev_status, void* stream) {
+  transmla_workspace_layout_t lay;
+  transmla_status_t st = transmla_workspace_layout(p, &lay);
+  if (st != TRANSMLA_OK) return st;
+  if (!q_nope || !w_uk || !cache || !page_table || !seqlens || !workspace) return TRANSMLA_ERR_NULL;
+  if (p->qk_rope_dim > 0 && !q_pe) return TRANSMLA_ERR_NULL;
+  if (!aligned(q_nope, 16) || !aligned(q_pe, 16) || !aligned(w_uk, 16) || !aligned(cache, 128) ||
+      !aligned(page_table, 4) || !aligned(seqlens, 4) || !aligned(workspace, kAlign) || !aligned(dev_status, 4))
+    return TRANSMLA_ERR_ALIGN;
+  if (workspace_bytes < lay.total_bytes) return TRANSMLA_ERR_WORKSPACE;
+  st = check_device(nullptr);
+  if (st != TRANSMLA_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  char* ws = static_cast<char*>(workspace);
+  auto* q_hat = reinterpret_cast<__nv_bfloat16*>(ws + lay.q_hat_offset);
+  auto* cum = reinterpret_cast<int32_t*>(ws + lay.cum_pages_offset);
+  auto* plan = reinterpret_cast<int32_t*>(ws + lay.plan_offset);
+  auto* po = reinterpret_cast<float*>(ws + lay.partial_o_offset);
+  auto* pl = reinterpret_cast<float*>(ws + lay.partial_lse_offset);
+  if (launch_plan(seqlens, p->batch, lay.num_partitions, cum, plan, s) != cudaSuccess) return TRANSMLA_ERR_CUDA;
+  if (launch_absorb(*p, static_cast<const __nv_bfloat16*>(q_nope), static_cast<const __nv_bfloat16*>(q_pe),
+                    static_cast<const __nv_bfloat16*>(w_uk), q_hat, s) != cudaSuccess)
+    return TRANSMLA_ERR_CUDA;
+  if (launch_decode_generic(*p, lay.num_partitions, q_hat, static_cast<const __nv_bfloat16*>(cache), page_table,
+                            seqlens, cum, plan, po, pl, dev_status, s) != cudaSuccess)
+    return TRANSMLA_ERR_CUDA;
+  return TRANSMLA_OK;
+}
+
+transmla_status_t transmla_mla_combine(const transmla_params_t* p, const void* workspace, size_t workspace_bytes,
+                                       const void* w_uv, void* out, float* lse_out, int32_t* dev_status,
+                                       void* stream) {
+  (void)dev_status;
+  transmla_workspace_layout_t lay;
+  transmla_status_t st = transmla_workspace_layout(p, &lay);
+  if (st != TRANSMLA_OK) return st;
+  if (!workspace || !w_uv || !out) return TRANSMLA_ERR_NULL;
+  if (!aligned(workspace, kAlign) || !aligned(w_uv, 16) || !aligned(out, 16) || !aligned(lse_out, 4))
+    return TRANSMLA_ERR_ALIGN;
+  if (workspace_bytes < lay.total_bytes) return TRANSMLA_ERR_WORKSPACE;
+  st = check_device(nullptr);
+  if (st != TRANSMLA_OK) return st;
+  const char* ws = static_cast<const char*>(workspace);
+  cudaError_t e = launch_combine(*p, lay.num_partitions, reinterpret_cast<const int32_t*>(ws + lay.cum_pages_offset),
+                                 reinterpret_cast<const float*>(ws + lay.partial_o_offset),
+                                 reinterpret_cast<const float*>(ws + lay.partial_lse_offset),
+                                 static_cast<const __nv_bfloat16*>(w_uv), static_cast<__nv_bfloat16*>(out), lse_out,
+                                 static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? TRANSMLA_OK : TRANSMLA_ERR_CUDA;
+}
+
+transmla_status_t transmla_validate_tables(const transmla_params_t* p, const int32_t* page_table,
+                                           const int32_t* seqlens) {
+  transmla_status_t st = check_shape(p, false);
+  if (st != TRANSMLA_OK) return st;
+  if (!page_table || !seqlens) return TRANSMLA_ERR_NULL;
+  std::vector<bool> used(static_cast<size_t>(p->num_pages), false);
+  for (int b = 0; b < p->batch; ++b) {
+    const int64_t L = seqlens[b];
+    if (L < 0 || L > static_cast<int64_t>(p->max_pages_per_seq) * kPage) return TRANSMLA_ERR_RANGE;
+    const int n = static_cast<int>((L + kPage - 1) / kPage);
+    for (int j = 0; j < n; ++j) {
+      const int32_t idx = page_table[static_cast<size_t>(b) * p->max_pages_per_seq + j];
+      if (idx < 0 || idx >= p->num_pages || used[idx]) return TRANSMLA_ERR_RANGE;
+      used[idx] = true;
+    }
+  }
+  return TRANSMLA_OK;
+}
+
+size_t transmla_step_staging_bytes(const transmla_params_t* p) {
+  if (check_shape(p, true) != TRANSMLA_OK) return 0;
+  const size_t B = p->batch, S = p->q_len, H = p->num_heads;
+  size_t off = 0;
+  off = round_up(off + B * S * p->hidden_dim * 2, kAlign);                 // x
+  off = round_up(off + B * S * H * p->qk_nope_dim * 2, kAlign);            // q_nope
+  off = round_up(off + B * S * H * p->qk_rope_dim * 2 + 16, kAlign);       // q_pe
+  off = round_up(off + B * p->max_pages_per_seq * 4, kAlign);              // page_table
+  off = round_up(off + B * 4, kAlign);                                     // seqlens
+  off = round_up(off + B * 4, kAlign);                                     // positions
+  off = round_up(off + B * S * H * p->v_dim * 2, kAlign);                  // out
+  off = round_up(off + B * S * H * 4, kAlign);                             // lse
+  off = round_up(off + 4, kAlign);                                         // device status word
+  return off;
+}
+
+transmla_status_t transmla_decode_step_host(const transmla_params_t* p, const void* h_x, const void* h_q_nope,
+                                            const void* h_q_pe, const int32_t* h_page_table,
+                                            const int32_t* h_seqlens, const void* w_dkv_kr, const void* w_uk,
+                                            const void* w_uv, void* cache, void* staging, size_t staging_bytes,
+                                            void* workspace, size_t workspace_bytes, void* h_out, float* h_lse,
+                                            int32_t* h_dev_status, void* stream) {
+  transmla_status_t st = check_shape(p, true);
+  if (st != TRANSMLA_OK) return st;
+  if (!h_x || !h_q_nope || !h_page_table || !h_seqlens || !w_dkv_kr || !w_uk || !w_uv || !cache || !staging ||
+      !workspace || !h_out)
+    return TRANSMLA_ERR_NULL;
+  if (p->qk_rope_dim > 0 && !h_q_pe) return TRANSMLA_ERR_NULL;
+  if (!aligned(staging, kAlign)) return TRANSMLA_ERR_ALIGN;
+  if (staging_bytes < transmla_step_staging_bytes(p)) return TRANSMLA_ERR_WORKSPACE;
+  st = transmla_validate_tables(p, h_page_table, h_seqlens);
+  if (st != TRANSMLA_OK) return st;
+  for (int b = 0; b < p->batch; ++b)
+    if (h_seqlens[b] < p->q_len) return TRANSMLA_ERR_RANGE;  // the step appends S tokens per sequence
+
+  const size_t B = p->batch, S = p->q_len, H = p->num_heads;
+  const size_t nx = B * S * p->hidden_dim * 2, nqn = B * S * H * p->qk_nope_dim * 2, nqp = B * S * H * p->qk_rope_dim * 2;
+  const size_t npt = B * p->max_pages_per_seq * 4, nout = B * S * H * p->v_dim * 2, nlse = B * S * H * 4;
+  char* base = static_cast<char*>(staging);
+  size_t off = 0;
+  char* d_x = base + off;    off = round_up(off + nx, kAlign);
+  char* d_qn = base + off;   off = round_up(off + nqn, kAlign);
+  char* d_qp = base + off;   off = round_up(off + nqp + 16, kAlign);
+  char* d_pt = base + off;   off = round_up(off + npt, kAlign);
+  char* d_sl = base + off;   off = round_up(off + B * 4, kAlign);
+  char* d_pos = base + off;  off = round_up(off + B * 4, kAlign);
+  char* d_out = base + off;  off = round_up(off + nout, kAlign);
+  char* d_lse = base + off;  off = round_up(off + nlse, kAlign);
+  char* d_st = base + off;
+
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  std::vector<int32_t> pos(B);
+  for (size_t b = 0; b < B; ++b) pos[b] = h_seqlens[b] - p->q_len;
+  bool ok = true;
+  ok &= cudaMemcpyAsync(d_x, h_x, nx, cudaMemcpyHostToDevice, s) == cudaSuccess;
+  ok &= cudaMemcpyAsync(d_qn, h_q_nope, nqn, cudaMemcpyHostToDevice, s) == cudaSuccess;
+  if (nqp) ok &= cudaMemcpyAsync(d_qp, h_q_pe, nqp, cudaMemcpyHostToDevice, s) == cudaSuccess;
+  ok &= cudaMemcpyAsync(d_pt, h_page_table, npt, cudaMemcpyHostToDevice, s) == cudaSuccess;
+  ok &= cudaMemcpyAsync(d_sl, h_seqlens, B * 4, cudaMemcpyHostToDevice, s) == cudaSuccess;
+  // pos is pageable host memory: the copy is staged by the runtime before the call returns
+  ok &= cudaMemcpyAsync(d_pos, pos.data(), B * 4, cudaMemcpyHostToDevice, s) == cudaSuccess;
+  ok &= cudaMemsetAsync(d_st, 0, 4, s) == cudaSuccess;
+  if (!ok) return TRANSMLA_ERR_CUDA;
+  auto* dst = reinterpret_cast<int32_t*>(d_st);
+  st = transmla_latent_append(p, d_x, w_dkv_kr, reinterpret_cast<int32_t*>(d_pos), reinterpret_cast<int32_t*>(d_pt),
+                              cache, dst, stream);
+  if (st != TRANSMLA_OK) return st;
+  st = transmla_mla_decode(p, d_qn, d_qp, w_uk, cache, reinterpret_cast<int32_t*>(d_pt),
+                           reinterpret_cast<int32_t*>(d_sl), workspace, workspace_bytes, dst, stream);
+  if (st != TRANSMLA_OK) return st;
+  st = transmla_mla_combine(p, workspace, workspace_bytes, w_uv, d_out, reinterpret_cast<float*>(d_lse), dst, stream);
+  if (st != TRANSMLA_OK) return st;
+  ok &= cudaMemcpyAsync(h_out, d_out, nout, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  if (h_lse) ok &= cudaMemcpyAsync(h_lse, d_lse, nlse, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  int32_t dev_word = 0;
+  ok &= cudaMemcpyAsync(&dev_word, d_st, 4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  ok &= cudaStreamSynchronize(s) == cudaSuccess;
+  if (h_dev_status) *h_dev_status = dev_word;
+  return ok ? TRANSMLA_OK : TRANSMLA_ERR_CUDA;
+}
+
+const char* transmla_status_string(transmla_status_t status) {
+  switch (status) {
+    case TRANSMLA_OK: return "ok";
+    case TRANSMLA_ERR_NULL: return "null pointer";
+    case TRANSMLA_ERR_ALIGN: return "misaligned pointer";
+    case TRANSMLA_ERR_SHAPE: return "unsupported shape";
+    case TRANSMLA_ERR_RANGE: return "sequence length or page index out of range";
+    case TRANSMLA_ERR_WORKSPACE: return "workspace too small";
+    case TRANSMLA_ERR_CUDA: return "CUDA call failed";
+    case TRANSMLA_ERR_ARCH: return "device is not sm_100";
+  }
+  return "unknown status";
+}
+
+}  // extern "C"

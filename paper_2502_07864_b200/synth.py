@@ -103,11 +103,12 @@ def make_decode_case(shape, seqlens, seed, pool_factor=1.2, device='cpu', nan_ta
 
 
 def make_append_case(shape, positions, seed, device='cpu'):
-    """Inputs of one append step: x [B, D] ~ N(0,1), w_dkv_kr [r+dR, D] ~ N(0, 1/sqrt(D)), bf16."""
+    """Inputs of one append step: x [B, S, D] ~ N(0,1), w_dkv_kr [r+dR, D] ~ N(0, 1/sqrt(D)), bf16;
+    positions [B] = position of each sequence's first new token."""
     g = _gen(seed, device)
     B = len(positions)
     return {
-        'x': _randn_bf16((B, shape.D), 1.0, g, device),
+        'x': _randn_bf16((B, shape.S, shape.D), 1.0, g, device),
         'w_dkv_kr': _randn_bf16((shape.row, shape.D), shape.D ** -0.5, g, device),
         'positions': torch.tensor([int(p) for p in positions], dtype=torch.int32, device=device),
     }

@@ -1,0 +1,80 @@
+"""GPU parity at the benchmark's full sizes, in the launch configuration the benchmark times.
+
+The oracle cannot finish every output of these cases in seconds, so it computes a seeded sample of
+(sequence, query position, head) outputs one by one; the CUDA results at those entries must meet the
+same tolerances as everywhere else.  Inputs are generated on the device with a seeded generator and
+only the sampled sequences' pages are copied back for the oracle.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2502_07864_b200 import synth
+from tests import gpu_util as gu
+from tests import lifts
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope='module', autouse=True)
+def _lib():
+    gu.ensure_built()
+
+
+def sub_case(case, seqs, P=64):
+    """The same inputs restricted to sequences `seqs`, with their pages packed into a small pool (CPU)."""
+    seqlens = [int(case['seqlens'][b]) for b in seqs]
+    n_pages = [(L + P - 1) // P for L in seqlens]
+    table = torch.full((len(seqs), max(max(n_pages), 1)), -1, dtype=torch.int32)
+    pages, k = [], 0
+    for i, b in enumerate(seqs):
+        idx = case['page_table'][b, :n_pages[i]].long()
+        pages.append(case['cache'][idx].cpu())
+        table[i, :n_pages[i]] = torch.arange(k, k + n_pages[i], dtype=torch.int32)
+        k += n_pages[i]
+    out = {k_: case[k_].cpu() for k_ in ('w_uk', 'w_uv')}
+    out.update(q_nope=case['q_nope'][seqs].cpu(), q_pe=case['q_pe'][seqs].cpu(),
+               cache=torch.cat(pages) if pages else case['cache'][:1].cpu(), page_table=table,
+               seqlens=torch.tensor(seqlens, dtype=torch.int32))
+    return out
+
+
+def check_sampled(shape, seqlens, seed, n_seq=3, n_heads=3):
+    scale = gu.mla_scale(shape)
+    case = synth.make_decode_case(shape, seqlens, seed, device='cuda')
+    out, lse, status, _, _ = gu.gpu_decode(shape, case, scale, G=0)
+    assert status == 0
+    assert torch.all(torch.isfinite(out.float()))
+    rng = np.random.default_rng(seed)
+    B = len(seqlens)
+    # always include the shortest and the longest sequence
+    seqs = sorted(set([int(np.argmin(seqlens)), int(np.argmax(seqlens))] +
+                      [int(b) for b in rng.choice(B, size=min(n_seq, B), replace=False)]))
+    sub = sub_case(case, seqs)
+    only = [(i, int(s), int(h)) for i in range(len(seqs)) for s in range(shape.S)
+            for h in rng.choice(shape.H, size=n_heads, replace=False)]
+    want, want_lse = gu.oracle_decode(shape, sub, scale, only=only)
+    got = lifts.f64(out[seqs])
+    got_lse = lifts.f64(lse[seqs])
+    idx = tuple(np.array(only).T)
+    gu.assert_close(got[idx], want[idx], f'sampled outputs B={B}')
+    gu.assert_lse_close(got_lse[idx], want_lse[idx], 'sampled lse')
+
+
+@pytest.mark.parametrize('B', [1, 4, 16, 64, 128])
+def test_llama_shape_batch_sweep_at_8k(B):
+    check_sampled(synth.LLAMA2_7B, [8192] * B, seed=3)
+
+
+def test_ragged_long_context_batch32():
+    seqlens = synth.uniform_seqlens(32, 1024, 32768, seed=4)
+    check_sampled(synth.LLAMA2_7B, seqlens, seed=4)
+
+
+def test_batch4_at_131072():
+    check_sampled(synth.LLAMA2_7B, [131072] * 4, seed=4, n_seq=1, n_heads=2)
+
+
+def test_qwen_like_two_query_positions_batch64():
+    seqlens = synth.uniform_seqlens(64, 2048, 8192, seed=5)
+    check_sampled(synth.QWEN25_72B, seqlens, seed=5)

@@ -1,0 +1,234 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle on the same seeded bytes.
+
+Tolerances (bf16 storage, fp32 accumulation): max-abs 2e-2 and relative L2 5e-3 on outputs;
+index paths (split plan, page slots, untouched cache bytes) bit-exact.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import mla_oracle as orc
+from paper_2502_07864_b200 import binding, synth
+from tests import gpu_util as gu
+from tests import lifts
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope='module', autouse=True)
+def _lib():
+    gu.ensure_built()
+
+
+def _run_and_compare(shape, seqlens, seed, G=0, scale=None, nan_tails=True, check_internals=False):
+    scale = scale if scale is not None else gu.mla_scale(shape)
+    case = synth.make_decode_case(shape, seqlens, seed, nan_tails=nan_tails)
+    out, lse, status, views, lay = gu.gpu_decode(shape, gu.to_dev(case), scale, G=G, want_views=check_internals)
+    assert status == 0
+    want_out, want_lse = gu.oracle_decode(shape, case, scale)
+    gu.assert_close(lifts.f64(out), want_out, f'out seqlens={seqlens} G={G}')
+    gu.assert_lse_close(lifts.f64(lse), want_lse, 'lse')
+    if check_internals:
+        c = lifts.case_f64(case)
+        # index path: bit-exact
+        cum, plan = orc.split_plan(seqlens, shape.page_size, lay.num_partitions)
+        assert np.array_equal(views['cum_pages'].cpu().numpy(), cum)
+        assert np.array_equal(views['plan'].cpu().numpy(), plan)
+        # absorbed queries: bf16 rounding of an fp32 sum
+        q_hat = orc.absorb(c['q_nope'], c['q_pe'], c['w_uk'])
+        got = lifts.f64(views['q_hat'])
+        assert np.all(np.abs(got - q_hat) <= 2.0 ** -7 * np.abs(q_hat) + 1e-3)
+        # per-segment partials against the oracle's own split of Eq. 9
+        B, S, H, r = len(seqlens), shape.S, shape.H, shape.r
+        po, pl = lifts.f64(views['partial_o']), lifts.f64(views['partial_lse'])
+        for (i, b, pb, pe, slot) in orc.plan_segments(cum, plan):
+            rows = orc.gather_latent(c['cache'], c['page_table'][b], int(seqlens[b]), shape.page_size)
+            n_vis = np.array([orc.visible_tokens(seqlens[b], S, s) for s in range(S) for _ in range(H)])
+            # the CUDA path rounds q_hat to bf16 before the contraction; the tolerance covers it
+            o, l = orc.decode_partial(q_hat[b].reshape(S * H, -1), n_vis, rows, r, scale,
+                                      pb * shape.page_size, pe * shape.page_size)
+            gu.assert_close(po[slot], o, f'partial_o slot {slot}')
+            gu.assert_lse_close(pl[slot], l, f'partial_lse slot {slot}')
+    return out, lse
+
+
+# ------------------------------------------------------------------ config 1: tiny, element by element
+@pytest.mark.parametrize('G', [0, 1, 2, 3, 7])
+def test_tiny_config_all_outputs_and_internals(G):
+    _run_and_compare(synth.TINY, [17, 64], seed=1, G=G, check_internals=True)
+
+
+def test_tiny_ragged_many_sequences():
+    _run_and_compare(synth.TINY, [1, 63, 64, 65, 128, 129, 200, 5, 700], seed=21, G=5, check_internals=True)
+
+
+@pytest.mark.parametrize('which', ['selector', 'replicated'])
+def test_gqa_lifts_reproduce_gqa(which):
+    # Sec. 4.1 / App. A.2.1: a GQA layer written as MLA gives the GQA output.
+    rng = np.random.default_rng(31)
+    if which == 'selector':
+        ref, m = lifts.selector_lift(rng, T=150)
+        shape = synth.MLAShape(H=8, dn=32, dR=0, dv=32, r=128, D=48)
+    else:
+        ref, m = lifts.replicated_lift(rng, T=150)
+        shape = synth.TINY
+    bf = lambda a: torch.tensor(np.nan_to_num(a, nan=0.0) if a.dtype.kind == 'f' else a)
+    case = {k: bf(m[k]).to(torch.bfloat16) for k in ('q_nope', 'q_pe', 'w_uk', 'w_uv')}
+    cache = torch.tensor(m['cache']).to(torch.bfloat16)        # NaN tails stay NaN
+    case.update(cache=cache, page_table=torch.tensor(m['page_table']), seqlens=torch.tensor(m['seqlens']))
+    out, lse, status, _, _ = gu.gpu_decode(shape, gu.to_dev(case), m['scale'], G=3)
+    assert status == 0
+    want, _ = gu.oracle_decode(shape, case, m['scale'])
+    gu.assert_close(lifts.f64(out), want, which)
+    # and, up to the bf16 rounding of the lifted inputs, the original GQA output
+    assert np.abs(lifts.f64(out)[0, 0] - ref).max() < 5e-2
+
+
+# ------------------------------------------------------------------ production shape, sizes spanning tiles + tails
+@pytest.mark.parametrize('seqlens,G', [([200, 327, 1000], 0), ([64 * 9], 4), ([1, 2, 63], 2), ([4096 + 17, 33], 13)])
+def test_llama_shape_medium(seqlens, G):
+    _run_and_compare(synth.LLAMA2_7B, seqlens, seed=2, G=G, check_internals=(len(seqlens) == 3 and G == 0))
+
+
+def test_qwen_shape_two_query_positions():
+    shape = synth.QWEN25_72B
+    _run_and_compare(shape, [130, 300, 2], seed=5, G=6, check_internals=True)
+
+
+def test_empty_sequences_and_short_pairs():
+    shape = synth.MLAShape(H=8, dn=32, dR=16, dv=32, r=64, D=256, S=2)
+    out, lse = _run_and_compare(shape, [0, 1, 2, 70], seed=7, G=3)
+    assert torch.all(out[0] == 0) and torch.all(torch.isneginf(lse[0]))
+    assert torch.all(out[1, 0] == 0) and torch.all(torch.isneginf(lse[1, 0]))   # L=1, S=2: query 0 sees nothing
+
+
+def test_results_are_bitwise_reproducible():
+    shape = synth.LLAMA2_7B
+    case = gu.to_dev(synth.make_decode_case(shape, [777, 1500], 8))
+    a = gu.gpu_decode(shape, case, gu.mla_scale(shape), G=9)
+    b = gu.gpu_decode(shape, case, gu.mla_scale(shape), G=9)
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+
+
+def test_page_permutation_gives_identical_bits():
+    shape = synth.LLAMA2_7B
+    case = synth.make_decode_case(shape, [500, 129], 9)
+    a = gu.gpu_decode(shape, gu.to_dev(case), gu.mla_scale(shape), G=5)
+    n = case['cache'].shape[0]
+    perm = torch.randperm(n, generator=torch.Generator().manual_seed(3))
+    case2 = dict(case)
+    case2['cache'] = torch.empty_like(case['cache'])
+    case2['cache'][perm] = case['cache']
+    pt = case['page_table'].long()
+    case2['page_table'] = torch.where(pt >= 0, perm[pt.clamp(min=0)], pt).to(torch.int32)
+    b = gu.gpu_decode(shape, gu.to_dev(case2), gu.mla_scale(shape), G=5)
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+
+
+def test_bad_page_index_is_reported_not_fatal():
+    shape = synth.TINY
+    case = synth.make_decode_case(shape, [100, 64], 10)
+    case['page_table'][0, 1] = case['cache'].shape[0] + 5
+    out, lse, status, _, _ = gu.gpu_decode(shape, gu.to_dev(case), 0.1, G=2)
+    assert status & 1
+    # the skipped page contributes nothing: same as a 64-token first sequence
+    case['seqlens'][0] = 64
+    want, _ = gu.oracle_decode(shape, case, 0.1)
+    gu.assert_close(lifts.f64(out), want, 'bad page skipped')
+
+
+def test_combine_alone_on_oracle_partials():
+    # feed the oracle's per-segment partials to the CUDA combine and compare with the oracle's result
+    shape = synth.TINY
+    seqlens = [300, 64, 0, 129]
+    scale = gu.mla_scale(shape)
+    case = synth.make_decode_case(shape, seqlens, 11)
+    c = lifts.case_f64(case)
+    G = 6
+    params = binding.make_params(shape, len(seqlens), case['cache'].shape[0], case['page_table'].shape[1], scale, G)
+    ws, lay = binding.alloc_workspace(params)
+    ws.zero_()
+    v = binding.workspace_views(params, ws, lay)
+    cum, plan = orc.split_plan(seqlens, 64, G)
+    v['cum_pages'].copy_(torch.tensor(cum))
+    v['partial_lse'].fill_(float('nan'))
+    v['partial_o'].fill_(float('nan'))
+    q_hat = orc.absorb(c['q_nope'], c['q_pe'], c['w_uk'])
+    for (i, b, pb, pe, slot) in orc.plan_segments(cum, plan):
+        rows = orc.gather_latent(c['cache'], c['page_table'][b], seqlens[b], 64)
+        o, l = orc.decode_partial(q_hat[b].reshape(shape.H, -1), np.full(shape.H, seqlens[b]), rows, shape.r, scale,
+                                  pb * 64, pe * 64)
+        v['partial_o'][slot] = torch.tensor(o, dtype=torch.float32)
+        v['partial_lse'][slot] = torch.tensor(l, dtype=torch.float32)
+    out = torch.empty(len(seqlens), 1, shape.H, shape.dv, dtype=torch.bfloat16, device='cuda')
+    lse = torch.empty(len(seqlens), 1, shape.H, dtype=torch.float32, device='cuda')
+    binding.transmla_mla_combine(params, ws, case['w_uv'].cuda(), out, lse)
+    torch.cuda.synchronize()
+    want, want_lse = gu.oracle_decode(shape, case, scale)
+    gu.assert_close(lifts.f64(out), want, 'combine')
+    gu.assert_lse_close(lifts.f64(lse), want_lse, 'combine lse')
+
+
+# ------------------------------------------------------------------ append
+@pytest.mark.parametrize('shape,positions', [(synth.TINY, [16, 63, 64, 0]), (synth.LLAMA2_7B, [8191, 0, 77, 131071]),
+                                             (synth.QWEN25_72B, [126, 63, 4000])])
+def test_append_values_slots_and_untouched_bytes(shape, positions):
+    B, S, P = len(positions), shape.S, shape.page_size
+    seqlens = [p + S for p in positions]
+    dc = synth.make_decode_case(shape, seqlens, 12)
+    ac = synth.make_append_case(shape, positions, 13)
+    x = ac['x']
+    params = binding.make_params(shape, B, dc['cache'].shape[0], dc['page_table'].shape[1], 1.0, num_partitions=1)
+    cache0 = dc['cache'].clone()
+    cache = dc['cache'].cuda()
+    status = torch.zeros(1, dtype=torch.int32, device='cuda')
+    binding.transmla_latent_append(params, x.cuda(), ac['w_dkv_kr'].cuda(), ac['positions'].cuda(),
+                                   dc['page_table'].cuda(), cache, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    got = cache.cpu()
+    want = lifts.f64(cache0)
+    touched = torch.zeros(cache0.shape[:2], dtype=torch.bool)
+    for s in range(S):
+        pos = [p + s for p in positions]
+        orc.latent_append(lifts.f64(x[:, s]), lifts.f64(ac['w_dkv_kr']), pos, dc['page_table'].numpy(), want, shape.r,
+                          page_size=P)
+        for b in range(B):
+            pg, off = orc.append_slot(dc['page_table'][b].numpy(), pos[b], P)       # slot: bit-exact index path
+            touched[pg, off] = True
+    g64 = lifts.f64(got)
+    t = touched.numpy()
+    assert np.all(np.abs(g64[t] - want[t]) <= 2.0 ** -7 * np.abs(want[t]) + 1e-3)
+    assert torch.equal(got.view(torch.int16)[~touched], cache0.view(torch.int16)[~touched])   # nothing else changed
+
+
+# ------------------------------------------------------------------ whole step from host buffers
+def test_decode_step_from_host_buffers():
+    shape = synth.LLAMA2_7B
+    seqlens = [300, 65, 1024]
+    B = len(seqlens)
+    scale = gu.mla_scale(shape)
+    dc = synth.make_decode_case(shape, seqlens, 15)
+    ac = synth.make_append_case(shape, [L - 1 for L in seqlens], 16)
+    params = binding.make_params(shape, B, dc['cache'].shape[0], dc['page_table'].shape[1], scale)
+    ws, _ = binding.alloc_workspace(params)
+    staging = torch.empty(binding.transmla_step_staging_bytes(params), dtype=torch.uint8, device='cuda')
+    pin = lambda t: t.contiguous().pin_memory()
+    h_out = torch.empty(B, 1, shape.H, shape.dv, dtype=torch.bfloat16).pin_memory()
+    h_lse = torch.empty(B, 1, shape.H, dtype=torch.float32).pin_memory()
+    cache = dc['cache'].cuda()
+    word = binding.transmla_decode_step_host(params, pin(ac['x']), pin(dc['q_nope']), pin(dc['q_pe']),
+                                             pin(dc['page_table']), pin(dc['seqlens']), ac['w_dkv_kr'].cuda(),
+                                             dc['w_uk'].cuda(), dc['w_uv'].cuda(), cache, staging, ws, h_out, h_lse)
+    assert word == 0
+    # oracle: append in fp64, round the new rows to bf16 as the cache stores them, then decode
+    want_cache = lifts.f64(dc['cache'])
+    orc.latent_append(lifts.f64(ac['x'][:, 0]), lifts.f64(ac['w_dkv_kr']), [L - 1 for L in seqlens], dc['page_table'].numpy(),
+                      want_cache, shape.r)
+    case = dict(dc)
+    case['cache'] = torch.tensor(want_cache).to(torch.bfloat16)
+    want, want_lse = gu.oracle_decode(shape, case, scale)
+    gu.assert_close(lifts.f64(h_out), want, 'host step')
+    gu.assert_lse_close(lifts.f64(h_lse), want_lse, 'host step lse')
