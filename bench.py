@@ -1,0 +1,320 @@
+#!/usr/bin/env python
+"""Benchmark of the absorbed-MLA decode step (append + absorb + split-KV decode + combine).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+One step = one pass of the whole path over one batch: every sequence appends its new token's
+latent and decodes over its cached tokens.  The default workload is the LLaMA-2-7B-converted
+shape (32 heads, latent 512 + rope 64, nope 128, v 128) at batch 16 x 8192 cached tokens.  With N
+GPUs every rank runs its own batch (sequences are independent; no collective on the data path),
+so the scaling is weak.  Rank 0 prints one JSON line.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = 'absorbed-MLA decode tokens/s and latent-cache HBM GB/s (% of 8 TB/s) at batch x 8K'
+NOMINAL_HBM_GBS = 8000.0
+KERNELS_PER_STEP = 6      # positions, append, plan, absorb, split-KV decode, combine
+
+
+def workloads():
+    from paper_2502_07864_b200 import synth
+    w = {}
+    for B in (1, 4, 16, 64, 128):
+        w[f'llama2-7b-mla_b{B}_8k'] = (synth.LLAMA2_7B, [8192] * B, 3)
+    w['llama2-7b-mla_b16_8k'] = (synth.LLAMA2_7B, [8192] * 16, 2)
+    w['llama2-7b-mla_ragged_b32'] = (synth.LLAMA2_7B, synth.uniform_seqlens(32, 1024, 32768, 4), 4)
+    w['llama2-7b-mla_b4_128k'] = (synth.LLAMA2_7B, [131072] * 4, 4)
+    w['qwen2.5-72b-mla_b64_s2'] = (synth.QWEN25_72B, synth.uniform_seqlens(64, 2048, 8192, 5), 5)
+    return w
+
+
+def measured_hbm_peak():
+    path = os.path.join(ROOT, 'MEASURED_PEAKS.json')
+    try:
+        return float(json.load(open(path))['hbm_gbs']), 'measured'
+    except Exception:
+        return 6650.0, 'fallback'
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ('clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,'
+              'clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap')
+
+    def __init__(self, index):
+        self.rows, self.proc = [], None
+        try:
+            self.proc = subprocess.Popen(['nvidia-smi', f'--query-gpu={self.FIELDS}', '--format=csv,noheader,nounits',
+                                          '-i', str(index), '-lms', '100'], stdout=subprocess.PIPE, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.perf_counter(), [c.strip() for c in line.split(',')]))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {'sm_mhz': None, 'sm_max_mhz': None, 'reasons': ['nvidia-smi unavailable']}
+        time.sleep(0.15)
+        self.proc.terminate()
+        rows = [r for (t, r) in self.rows if t0 <= t <= t1 + 0.15] or [r for (_, r) in self.rows[-3:]]
+        sm, mx, reasons = [], None, set()
+        for r in rows:
+            try:
+                sm.append(float(r[0])); mx = float(r[1])
+            except Exception:
+                continue
+            for name, v in zip(('hw_slowdown', 'hw_thermal_slowdown', 'sw_thermal_slowdown', 'sw_power_cap'), r[2:6]):
+                if v.lower().startswith('active'):
+                    reasons.add(name)
+        return {'sm_mhz': statistics.median(sm) if sm else None, 'sm_max_mhz': mx, 'reasons': sorted(reasons),
+                'samples': len(sm)}
+
+
+def oracle_sample(shape, seqlens, seed, n_seq):
+    """Inputs of the first n_seq sequences of the workload, on the CPU, as float64 numpy."""
+    import torch
+    from paper_2502_07864_b200 import synth
+    case = synth.make_decode_case(shape, seqlens[:n_seq], seed, device='cpu')
+    return {k: (v.to(torch.float64).numpy() if v.is_floating_point() else v.numpy()) for k, v in case.items()}
+
+
+def time_oracle(shape, c, scale):
+    from oracle import mla_oracle as orc
+    t0 = time.perf_counter()
+    orc.mla_decode_mha_form(c['q_nope'], c['q_pe'], c['w_uk'], c['w_uv'], c['cache'], c['page_table'], c['seqlens'],
+                            scale, page_size=shape.page_size)
+    return time.perf_counter() - t0
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p['num_threads'] for p in threadpool_info() if p.get('user_api') == 'blas']
+        return max(n) if n else os.cpu_count()
+    except Exception:
+        return os.cpu_count()
+
+
+def cpu_baseline(shape, seqlens, seed, scale, budget_s=15.0):
+    """The fp64 oracle, as it stands, on a bounded sample: whole sequences of the workload, all heads."""
+    c1 = oracle_sample(shape, seqlens, seed, 1)
+    t1 = time_oracle(shape, c1, scale)
+    n = int(max(1, min(len(seqlens), budget_s // max(t1, 1e-3))))
+    if n > 1:
+        c = oracle_sample(shape, seqlens, seed, n)
+        t = time_oracle(shape, c, scale)
+    else:
+        t = t1
+    return {'value': n * shape.S / t, 'unit': 'tokens/s', 'cores': blas_threads(), 'kind': 'oracle',
+            'sample': f'first {n} of {len(seqlens)} sequences, all {shape.H} heads, all cached tokens; {t:.1f} s'}
+
+
+def run_reference(args, name, shape, seqlens, seed):
+    """The oracle as the reference arm: every step decodes a bounded sample of the workload on the host.
+
+    The sample is the first sequence of the workload, all its cached tokens, and as many heads as fit
+    a per-step time budget chosen so that the whole run ends within a few minutes; a step that does
+    n of the H heads of one token counts as n/H tokens.
+    """
+    rank = int(os.environ.get('RANK', '0'))
+    if rank != 0:
+        return
+    from oracle import mla_oracle as orc
+    scale = (shape.dn + shape.dR) ** -0.5
+    c = oracle_sample(shape, seqlens, seed, 1)
+
+    def run(only):
+        t0 = time.perf_counter()
+        orc.mla_decode_mha_form(c['q_nope'], c['q_pe'], c['w_uk'], c['w_uv'], c['cache'], c['page_table'],
+                                c['seqlens'], scale, page_size=shape.page_size, only=only)
+        return time.perf_counter() - t0
+    run([(0, 0, 0)])
+    t_head = run([(0, 0, 0)])
+    budget = min(1.0, 150.0 / max(args.steps + args.warmup, 1))
+    n_heads = int(max(1, min(shape.H, budget // max(t_head, 1e-4))))
+    only = [(0, s, h) for s in range(shape.S) for h in range(n_heads)]
+    for _ in range(args.warmup):
+        run(only)
+    t = sum(run(only) for _ in range(args.steps))
+    tokens_per_step = shape.S * n_heads / shape.H
+    value = args.steps * tokens_per_step / t
+    sample = f'1 of {len(seqlens)} sequences ({seqlens[0]} cached tokens), {n_heads} of {shape.H} heads per step'
+    print(json.dumps({
+        'impl': 'reference', 'metric': METRIC, 'value': value, 'unit': 'tokens/s', 'n_gpus': args.gpus,
+        'steps': args.steps, 'warmup': args.warmup, 'ms_per_step': 1e3 * t / args.steps, 'higher_is_better': True,
+        'scaling': 'weak', 'vs_baseline': None, 'dtype': 'f64', 'data': 'synthetic',
+        'config': {'workload': name, 'sample': sample},
+        'cpu_baseline': {'value': value, 'unit': 'tokens/s', 'cores': blas_threads(), 'kind': 'oracle', 'sample': sample},
+        'e2e': {'value': value, 'unit': 'tokens/s', 'h2d_bytes_per_step': 0, 'd2h_bytes_per_step': 0},
+    }))
+
+
+def run_ours(args, name, shape, seqlens, seed):
+    import torch
+    import torch.distributed as dist
+    from paper_2502_07864_b200 import binding, build, synth
+
+    rank = int(os.environ.get('RANK', '0'))
+    world = int(os.environ.get('WORLD_SIZE', '1'))
+    local = int(os.environ.get('LOCAL_RANK', '0'))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group('nccl', device_id=torch.device('cuda', local))
+    if rank == 0:
+        build.build()
+    if world > 1:
+        dist.barrier()
+    binding.lib()          # raises if the CUDA library is missing: there is no other path
+
+    B, S, H = len(seqlens), shape.S, shape.H
+    scale = (shape.dn + shape.dR) ** -0.5
+    n_copies = args.cache_copies
+    dc = synth.make_decode_case(shape, seqlens, seed + 100 * rank, device='cuda')
+    ac = synth.make_append_case(shape, [L - S for L in seqlens], seed + 100 * rank + 1, device='cuda')
+    caches = [dc['cache']] + [dc['cache'].clone() for _ in range(n_copies - 1)]
+    params = binding.make_params(shape, B, dc['cache'].shape[0], dc['page_table'].shape[1], scale)
+    ws, lay = binding.alloc_workspace(params)
+    out = torch.empty(B, S, H, shape.dv, dtype=torch.bfloat16, device='cuda')
+    lse = torch.empty(B, S, H, dtype=torch.float32, device='cuda')
+    status = torch.zeros(1, dtype=torch.int32, device='cuda')
+    pos = torch.empty(B, dtype=torch.int32, device='cuda')
+    stream = torch.cuda.current_stream()
+
+    def step(i, ev=None):
+        if ev is not None:
+            binding.transmla_profile_decode_kernel(ev[0], ev[1])
+        binding.transmla_decode_step(params, ac['x'], dc['q_nope'], dc['q_pe'], dc['page_table'], dc['seqlens'],
+                                     ac['w_dkv_kr'], dc['w_uk'], dc['w_uv'], caches[i % n_copies], pos, ws, out, lse,
+                                     status, stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    barrier()
+
+    kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for a, b_ in kev:       # create the underlying CUDA events before handing them to the library
+        a.record(stream); b_.record(stream)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local) if rank == 0 else None
+    barrier()
+    t0 = time.perf_counter()
+    e0.record(stream)
+    for i in range(args.steps):
+        step(i, kev[i])
+    e1.record(stream)
+    barrier()
+    t1 = time.perf_counter()
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop(t0, t1) if sampler else None
+    kernel_ms = statistics.mean(a.elapsed_time(b_) for a, b_ in kev)
+    assert int(status.item()) == 0, 'device status word set'
+
+    # end to end through the host-buffer entry point: pinned host inputs, result read back every step
+    staging = torch.empty(binding.transmla_step_staging_bytes(params), dtype=torch.uint8, device='cuda')
+    pin = lambda t: t.cpu().contiguous().pin_memory()
+    h = {k: pin(v) for k, v in (('x', ac['x']), ('q_nope', dc['q_nope']), ('q_pe', dc['q_pe']),
+                                ('page_table', dc['page_table']), ('seqlens', dc['seqlens']))}
+    h_out = torch.empty(B, S, H, shape.dv, dtype=torch.bfloat16).pin_memory()
+    h_lse = torch.empty(B, S, H, dtype=torch.float32).pin_memory()
+
+    def host_step(i):
+        return binding.transmla_decode_step_host(params, h['x'], h['q_nope'], h['q_pe'], h['page_table'], h['seqlens'],
+                                                 ac['w_dkv_kr'], dc['w_uk'], dc['w_uv'], caches[i % n_copies], staging,
+                                                 ws, h_out, h_lse, stream)
+    for i in range(3):
+        host_step(i)
+    barrier()
+    t2 = time.perf_counter()
+    for i in range(args.steps):
+        host_step(i)
+    barrier()
+    e2e_s = time.perf_counter() - t2
+    h2d = sum(v.numel() * v.element_size() for v in h.values())
+    d2h = h_out.numel() * 2 + h_lse.numel() * 4 + 4
+
+    times = torch.tensor([ms_total, e2e_s * 1e3], dtype=torch.float64, device='cuda')
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    ms_total, e2e_ms = (float(v) for v in times.tolist())
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    tokens_per_step = B * S * world
+    ms_step = ms_total / args.steps
+    cache_bytes = sum(seqlens) * shape.row * 2                       # live latent rows, read once
+    q_hat_bytes = B * S * H * shape.row * 2
+    algo_bytes = cache_bytes + q_hat_bytes                           # per split-KV launch
+    achieved = algo_bytes / (kernel_ms * 1e-3) / 1e9
+    peak, peak_kind = measured_hbm_peak()
+    traffic = None
+    line = {
+        'metric': METRIC, 'value': tokens_per_step / (ms_step * 1e-3), 'unit': 'tokens/s', 'n_gpus': world,
+        'steps': args.steps, 'warmup': max(args.warmup, 3), 'ms_per_step': ms_step, 'higher_is_better': True,
+        'scaling': 'weak', 'vs_baseline': None, 'dtype': 'bf16', 'data': 'synthetic',
+        'config': {'workload': name, 'batch_per_gpu': B, 'q_len': S, 'heads': H, 'latent': shape.r, 'rope': shape.dR,
+                   'cached_tokens_per_gpu': sum(seqlens), 'page_size': shape.page_size,
+                   'num_partitions': lay.num_partitions,
+                   'l2': f'cache rotates over {n_copies} copies ({n_copies * cache_bytes / 1e6:.0f} MB) between steps',
+                   'parallelism': f'replicas x{world}, no data-path collective'},
+        'cache_gbs': world * cache_bytes / (ms_step * 1e-3) / 1e9,
+        'cache_gbs_pct_of_8tbs': 100.0 * cache_bytes / (ms_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+        'decode_kernel_us': kernel_ms * 1e3,
+        'roofline': {'bound': 'hbm', 'achieved': achieved, 'peak': peak, 'unit': 'GB/s', 'frac': achieved / peak,
+                     'peak_kind': f'{peak_kind} copy bandwidth', 'frac_of_8tbs': achieved / NOMINAL_HBM_GBS,
+                     'kernel': 'split-KV decode', 'algorithmic_bytes_per_launch': algo_bytes, 'traffic': traffic},
+        'e2e': {'value': tokens_per_step / (e2e_ms * 1e-3 / args.steps), 'unit': 'tokens/s',
+                'h2d_bytes_per_step': h2d, 'd2h_bytes_per_step': d2h, 'ms_per_step': e2e_ms / args.steps},
+        'gpu_launches': KERNELS_PER_STEP * args.steps,
+        'clocks': clocks,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        line['cpu_baseline'] = cpu_baseline(shape, seqlens, seed, scale)
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument('--gpus', type=int, default=1)
+    ap.add_argument('--steps', type=int, default=200)
+    ap.add_argument('--warmup', type=int, default=10)
+    ap.add_argument('--impl', default='ours', choices=['ours', 'reference'])
+    ap.add_argument('--workload', default='llama2-7b-mla_b16_8k')
+    ap.add_argument('--cache-copies', type=int, default=4)
+    ap.add_argument('--no-cpu-baseline', action='store_true')
+    args = ap.parse_args()
+    w = workloads()
+    if args.workload not in w:
+        sys.exit(f'unknown workload {args.workload}; choose from {sorted(w)}')
+    shape, seqlens, seed = w[args.workload]
+    if args.impl == 'reference':
+        run_reference(args, args.workload, shape, seqlens, seed)
+    else:
+        run_ours(args, args.workload, shape, seqlens, seed)
+
+
+if __name__ == '__main__':
+    main()

@@ -157,15 +157,27 @@ transmla_status_t transmla_validate_tables(const transmla_params_t* params /* ho
                                            const int32_t* page_table /* host */,
                                            const int32_t* seqlens /* host */);
 
+/* One whole decode step on device buffers: append the S new tokens of every sequence at positions
+ * L_b - S .. L_b - 1 (transmla_latent_append with positions[b] = L_b - S, computed on the device),
+ * then transmla_mla_decode and transmla_mla_combine.  Same arguments and rules as those three calls;
+ * `positions_scratch` is a device int32 [B] buffer the call overwrites.  Every sequence needs
+ * L_b >= S. */
+transmla_status_t transmla_decode_step(const transmla_params_t* params /* host */, const void* x,
+                                       const void* q_nope, const void* q_pe, const int32_t* page_table,
+                                       const int32_t* seqlens, const void* w_dkv_kr, const void* w_uk,
+                                       const void* w_uv, void* cache, int32_t* positions_scratch,
+                                       void* workspace, size_t workspace_bytes, void* out, float* lse_out,
+                                       int32_t* dev_status, void* stream);
+
 /* Bytes of device staging transmla_decode_step_host needs for `params`. */
 size_t transmla_step_staging_bytes(const transmla_params_t* params /* host */);
 
-/* One whole decode step driven from host buffers: validates the tables, copies this step's inputs to
- * the device (x, q_nope, q_pe, page_table, seqlens), appends the S new tokens of every sequence at
- * positions L_b - S .. L_b - 1, runs decode and combine, copies `out` (and `lse` if not NULL) back
- * and waits for `stream`.  Weights and the cache stay resident on the device.  Host buffers should
- * be pinned for the copies to be asynchronous.  Returns the first error, or TRANSMLA_OK;
- * `*h_dev_status` (host, may be NULL) receives the device status word.
+/* One whole decode step driven from host buffers: validates the tables on the host, copies this
+ * step's inputs to the device (x, q_nope, q_pe, page_table, seqlens), runs transmla_decode_step,
+ * copies `out` (and `lse` if not NULL) back and waits for `stream`.  Weights and the cache stay
+ * resident on the device.  Host buffers should be pinned for the copies to be asynchronous.  Uses
+ * host heap memory for the validation; allocates no device memory.  Returns the first error, or
+ * TRANSMLA_OK; `*h_dev_status` (host, may be NULL) receives the device status word.
  *   h_x [B,S,D], h_q_nope [B,S,H,dn], h_q_pe [B,S,H,dR], h_page_table, h_seqlens : host
  *   w_dkv_kr, w_uk, w_uv, cache, staging, workspace                              : device
  *   h_out [B,S,H,dv] bf16, h_lse [B,S,H] fp32 or NULL                            : host */
@@ -176,6 +188,11 @@ transmla_status_t transmla_decode_step_host(const transmla_params_t* params, con
                                             void* cache, void* staging, size_t staging_bytes,
                                             void* workspace, size_t workspace_bytes, void* h_out,
                                             float* h_lse, int32_t* h_dev_status, void* stream);
+
+/* Timing hook: the next transmla_mla_decode issued by the calling thread records `start_event`
+ * immediately before and `stop_event` immediately after its split-KV kernel on that call's stream
+ * (both cudaEvent_t passed as void*; NULL, NULL clears the hook).  The hook is consumed by that call. */
+void transmla_profile_decode_kernel(void* start_event, void* stop_event);
 
 /* Human-readable name of a status code (static storage). */
 const char* transmla_status_string(transmla_status_t status);

@@ -13,7 +13,7 @@ _LIB_PATH = os.path.join(_HERE, 'libtransmla.so')
 
 EXPORTS = ('transmla_workspace_layout', 'transmla_latent_append', 'transmla_mla_decode', 'transmla_mla_combine',
            'transmla_validate_tables', 'transmla_step_staging_bytes', 'transmla_decode_step_host',
-           'transmla_status_string')
+           'transmla_decode_step', 'transmla_profile_decode_kernel', 'transmla_status_string')
 
 
 class Params(ctypes.Structure):
@@ -57,10 +57,14 @@ def lib():
         L.transmla_step_staging_bytes.restype = sz
         L.transmla_decode_step_host.argtypes = [pp, vp, vp, vp, i32p, i32p, vp, vp, vp, vp, vp, sz, vp, sz, vp, vp,
                                                 i32p, vp]
+        L.transmla_decode_step.argtypes = [pp, vp, vp, vp, i32p, i32p, vp, vp, vp, vp, i32p, vp, sz, vp, vp, i32p, vp]
+        L.transmla_profile_decode_kernel.argtypes = [vp, vp]
+        L.transmla_profile_decode_kernel.restype = None
         L.transmla_status_string.argtypes = [ctypes.c_int]
         L.transmla_status_string.restype = ctypes.c_char_p
         for name in EXPORTS:
-            if name not in ('transmla_step_staging_bytes', 'transmla_status_string'):
+            if name not in ('transmla_step_staging_bytes', 'transmla_status_string',
+                            'transmla_profile_decode_kernel'):
                 getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -140,6 +144,22 @@ def transmla_decode_step_host(params, h_x, h_q_nope, h_q_pe, h_page_table, h_seq
         _ptr(h_out), _ptr(h_lse), ctypes.cast(ctypes.byref(word), ctypes.c_void_p), _stream(stream)),
         'transmla_decode_step_host')
     return word.value
+
+
+def transmla_decode_step(params, x, q_nope, q_pe, page_table, seqlens, w_dkv_kr, w_uk, w_uv, cache,
+                         positions_scratch, workspace, out, lse_out=None, dev_status=None, stream=None):
+    _check(lib().transmla_decode_step(
+        ctypes.byref(params), _ptr(x), _ptr(q_nope), _ptr(q_pe), _ptr(page_table), _ptr(seqlens), _ptr(w_dkv_kr),
+        _ptr(w_uk), _ptr(w_uv), _ptr(cache), _ptr(positions_scratch), _ptr(workspace),
+        workspace.numel() * workspace.element_size(), _ptr(out), _ptr(lse_out), _ptr(dev_status), _stream(stream)),
+        'transmla_decode_step')
+
+
+def transmla_profile_decode_kernel(start_event, stop_event):
+    """torch.cuda.Event objects (timing enabled, already created by a record) or None, None."""
+    a = ctypes.c_void_p(0 if start_event is None else start_event.cuda_event)
+    b = ctypes.c_void_p(0 if stop_event is None else stop_event.cuda_event)
+    lib().transmla_profile_decode_kernel(a, b)
 
 
 # -------- conveniences built only from the calls above (device-memory plumbing, no arithmetic)

@@ -43,9 +43,21 @@ transmla_status_t check_device(int* sm_count) {
   return TRANSMLA_OK;
 }
 
+thread_local cudaEvent_t tl_prof_start = nullptr, tl_prof_stop = nullptr;
+
+__global__ void positions_kernel(const int32_t* __restrict__ seqlens, int32_t* __restrict__ positions, int B, int S) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b < B) positions[b] = seqlens[b] - S;
+}
+
 }  // namespace
 
 extern "C" {
+
+void transmla_profile_decode_kernel(void* start_event, void* stop_event) {
+  tl_prof_start = static_cast<cudaEvent_t>(start_event);
+  tl_prof_stop = static_cast<cudaEvent_t>(stop_event);
+}
 
 transmla_status_t transmla_workspace_layout(const transmla_params_t* p, transmla_workspace_layout_t* out) {
   if (out == nullptr) return TRANSMLA_ERR_NULL;
@@ -118,9 +130,13 @@ transmla_status_t transmla_mla_decode(const transmla_params_t* p, const void* q_
   if (launch_absorb(*p, static_cast<const __nv_bfloat16*>(q_nope), static_cast<const __nv_bfloat16*>(q_pe),
                     static_cast<const __nv_bfloat16*>(w_uk), q_hat, s) != cudaSuccess)
     return TRANSMLA_ERR_CUDA;
+  cudaEvent_t ev0 = tl_prof_start, ev1 = tl_prof_stop;
+  tl_prof_start = tl_prof_stop = nullptr;
+  if (ev0 != nullptr && cudaEventRecord(ev0, s) != cudaSuccess) return TRANSMLA_ERR_CUDA;
   if (launch_decode_generic(*p, lay.num_partitions, q_hat, static_cast<const __nv_bfloat16*>(cache), page_table,
                             seqlens, cum, plan, po, pl, dev_status, s) != cudaSuccess)
     return TRANSMLA_ERR_CUDA;
+  if (ev1 != nullptr && cudaEventRecord(ev1, s) != cudaSuccess) return TRANSMLA_ERR_CUDA;
   return TRANSMLA_OK;
 }
 
@@ -163,6 +179,30 @@ transmla_status_t transmla_validate_tables(const transmla_params_t* p, const int
     }
   }
   return TRANSMLA_OK;
+}
+
+transmla_status_t transmla_decode_step(const transmla_params_t* p, const void* x, const void* q_nope,
+                                       const void* q_pe, const int32_t* page_table, const int32_t* seqlens,
+                                       const void* w_dkv_kr, const void* w_uk, const void* w_uv, void* cache,
+                                       int32_t* positions_scratch, void* workspace, size_t workspace_bytes,
+                                       void* out, float* lse_out, int32_t* dev_status, void* stream) {
+  transmla_status_t st = check_shape(p, true);
+  if (st != TRANSMLA_OK) return st;
+  if (!positions_scratch || !seqlens) return TRANSMLA_ERR_NULL;
+  if (!aligned(positions_scratch, 4) || !aligned(seqlens, 4)) return TRANSMLA_ERR_ALIGN;
+  if (!x || !w_dkv_kr || !page_table || !cache || !q_nope || !w_uk || !workspace || !w_uv || !out)
+    return TRANSMLA_ERR_NULL;
+  st = check_device(nullptr);
+  if (st != TRANSMLA_OK) return st;
+  positions_kernel<<<(p->batch + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      seqlens, positions_scratch, p->batch, p->q_len);
+  if (cudaGetLastError() != cudaSuccess) return TRANSMLA_ERR_CUDA;
+  st = transmla_latent_append(p, x, w_dkv_kr, positions_scratch, page_table, cache, dev_status, stream);
+  if (st != TRANSMLA_OK) return st;
+  st = transmla_mla_decode(p, q_nope, q_pe, w_uk, cache, page_table, seqlens, workspace, workspace_bytes, dev_status,
+                           stream);
+  if (st != TRANSMLA_OK) return st;
+  return transmla_mla_combine(p, workspace, workspace_bytes, w_uv, out, lse_out, dev_status, stream);
 }
 
 size_t transmla_step_staging_bytes(const transmla_params_t* p) {
@@ -216,26 +256,18 @@ transmla_status_t transmla_decode_step_host(const transmla_params_t* p, const vo
   char* d_st = base + off;
 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  std::vector<int32_t> pos(B);
-  for (size_t b = 0; b < B; ++b) pos[b] = h_seqlens[b] - p->q_len;
   bool ok = true;
   ok &= cudaMemcpyAsync(d_x, h_x, nx, cudaMemcpyHostToDevice, s) == cudaSuccess;
   ok &= cudaMemcpyAsync(d_qn, h_q_nope, nqn, cudaMemcpyHostToDevice, s) == cudaSuccess;
   if (nqp) ok &= cudaMemcpyAsync(d_qp, h_q_pe, nqp, cudaMemcpyHostToDevice, s) == cudaSuccess;
   ok &= cudaMemcpyAsync(d_pt, h_page_table, npt, cudaMemcpyHostToDevice, s) == cudaSuccess;
   ok &= cudaMemcpyAsync(d_sl, h_seqlens, B * 4, cudaMemcpyHostToDevice, s) == cudaSuccess;
-  // pos is pageable host memory: the copy is staged by the runtime before the call returns
-  ok &= cudaMemcpyAsync(d_pos, pos.data(), B * 4, cudaMemcpyHostToDevice, s) == cudaSuccess;
   ok &= cudaMemsetAsync(d_st, 0, 4, s) == cudaSuccess;
   if (!ok) return TRANSMLA_ERR_CUDA;
   auto* dst = reinterpret_cast<int32_t*>(d_st);
-  st = transmla_latent_append(p, d_x, w_dkv_kr, reinterpret_cast<int32_t*>(d_pos), reinterpret_cast<int32_t*>(d_pt),
-                              cache, dst, stream);
-  if (st != TRANSMLA_OK) return st;
-  st = transmla_mla_decode(p, d_qn, d_qp, w_uk, cache, reinterpret_cast<int32_t*>(d_pt),
-                           reinterpret_cast<int32_t*>(d_sl), workspace, workspace_bytes, dst, stream);
-  if (st != TRANSMLA_OK) return st;
-  st = transmla_mla_combine(p, workspace, workspace_bytes, w_uv, d_out, reinterpret_cast<float*>(d_lse), dst, stream);
+  st = transmla_decode_step(p, d_x, d_qn, d_qp, reinterpret_cast<int32_t*>(d_pt), reinterpret_cast<int32_t*>(d_sl),
+                            w_dkv_kr, w_uk, w_uv, cache, reinterpret_cast<int32_t*>(d_pos), workspace, workspace_bytes,
+                            d_out, reinterpret_cast<float*>(d_lse), dst, stream);
   if (st != TRANSMLA_OK) return st;
   ok &= cudaMemcpyAsync(h_out, d_out, nout, cudaMemcpyDeviceToHost, s) == cudaSuccess;
   if (h_lse) ok &= cudaMemcpyAsync(h_lse, d_lse, nlse, cudaMemcpyDeviceToHost, s) == cudaSuccess;

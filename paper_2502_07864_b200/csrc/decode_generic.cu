@@ -96,6 +96,9 @@ decode_generic_kernel(const __nv_bfloat16* __restrict__ q_hat, const __nv_bfloat
 
     for (int pj = pg_lo; pj < pg_hi; ++pj) {
       const int stage = (pj - pg_lo) & 1;
+      const int idx_cur = page_table[static_cast<size_t>(b) * max_pages + pj];
+      // tokens of a page whose index is out of range are masked like tokens beyond the sequence
+      const int tok_end = (idx_cur >= 0 && idx_cur < num_pages) ? n_vis - pj * kPage : 0;
       cp_async_wait<0>();
       __syncthreads();  // page pj (and, first time, the queries) landed; everyone is done with the other stage
       if (pj + 1 < pg_hi) { load_page(pj + 1, stage ^ 1); cp_async_commit(); }
@@ -161,7 +164,7 @@ decode_generic_kernel(const __nv_bfloat16* __restrict__ q_hat, const __nv_bfloat
           float v = 0.f;
 #pragma unroll
           for (int w = 0; w < 4; ++w) v += s_s[(w * kRowBlock + srow) * SP + tok];
-          v = (pj * kPage + tok < n_vis) ? v * scale_log2 : -INFINITY;
+          v = (tok < tok_end) ? v * scale_log2 : -INFINITY;
           z[j] = v;
           tmax = fmaxf(tmax, v);
         }
