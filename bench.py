@@ -24,7 +24,7 @@ if ROOT not in sys.path:
 
 METRIC = 'absorbed-MLA decode tokens/s and latent-cache HBM GB/s (% of 8 TB/s) at batch x 8K'
 NOMINAL_HBM_GBS = 8000.0
-KERNELS_PER_STEP = 6      # positions, append, plan, absorb, split-KV decode, combine
+KERNELS_PER_STEP = 3      # prologue (append + absorb + plan), split-KV decode, combine
 
 
 def workloads():
@@ -192,14 +192,13 @@ def run_ours(args, name, shape, seqlens, seed):
     out = torch.empty(B, S, H, shape.dv, dtype=torch.bfloat16, device='cuda')
     lse = torch.empty(B, S, H, dtype=torch.float32, device='cuda')
     status = torch.zeros(1, dtype=torch.int32, device='cuda')
-    pos = torch.empty(B, dtype=torch.int32, device='cuda')
     stream = torch.cuda.current_stream()
 
     def step(i, ev=None):
         if ev is not None:
             binding.transmla_profile_decode_kernel(ev[0], ev[1])
         binding.transmla_decode_step(params, ac['x'], dc['q_nope'], dc['q_pe'], dc['page_table'], dc['seqlens'],
-                                     ac['w_dkv_kr'], dc['w_uk'], dc['w_uv'], caches[i % n_copies], pos, ws, out, lse,
+                                     ac['w_dkv_kr'], dc['w_uk'], dc['w_uv'], caches[i % n_copies], ws, out, lse,
                                      status, stream)
 
     def barrier():

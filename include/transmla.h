@@ -69,7 +69,7 @@ typedef struct {
   float rope_theta;          /* RoPE base, 10000 in Eq. 1 */
 } transmla_params_t;
 
-/* Supported (r, dR) pairs: (512, 64), (128, 0), (64, 16).  dn, dv: multiples of 8 up to 256.
+/* Supported (r, dR) pairs: (512, 64), (128, 0), (64, 16).  dn: multiple of 16, dv: multiple of 8, both up to 256; D: multiple of 128.
  * S*H <= 1024.  page_size == 64. */
 
 /* Byte offsets of the regions inside the workspace that carries results from
@@ -158,16 +158,15 @@ transmla_status_t transmla_validate_tables(const transmla_params_t* params /* ho
                                            const int32_t* seqlens /* host */);
 
 /* One whole decode step on device buffers: append the S new tokens of every sequence at positions
- * L_b - S .. L_b - 1 (transmla_latent_append with positions[b] = L_b - S, computed on the device),
- * then transmla_mla_decode and transmla_mla_combine.  Same arguments and rules as those three calls;
- * `positions_scratch` is a device int32 [B] buffer the call overwrites.  Every sequence needs
- * L_b >= S. */
+ * L_b - S .. L_b - 1 (what transmla_latent_append does with positions[b] = L_b - S), then what
+ * transmla_mla_decode and transmla_mla_combine do, in three launches.  Same arguments and rules as
+ * those three calls.  Every sequence needs L_b >= S. */
 transmla_status_t transmla_decode_step(const transmla_params_t* params /* host */, const void* x,
                                        const void* q_nope, const void* q_pe, const int32_t* page_table,
                                        const int32_t* seqlens, const void* w_dkv_kr, const void* w_uk,
-                                       const void* w_uv, void* cache, int32_t* positions_scratch,
-                                       void* workspace, size_t workspace_bytes, void* out, float* lse_out,
-                                       int32_t* dev_status, void* stream);
+                                       const void* w_uv, void* cache, void* workspace,
+                                       size_t workspace_bytes, void* out, float* lse_out, int32_t* dev_status,
+                                       void* stream);
 
 /* Bytes of device staging transmla_decode_step_host needs for `params`. */
 size_t transmla_step_staging_bytes(const transmla_params_t* params /* host */);

@@ -57,7 +57,7 @@ def lib():
         L.transmla_step_staging_bytes.restype = sz
         L.transmla_decode_step_host.argtypes = [pp, vp, vp, vp, i32p, i32p, vp, vp, vp, vp, vp, sz, vp, sz, vp, vp,
                                                 i32p, vp]
-        L.transmla_decode_step.argtypes = [pp, vp, vp, vp, i32p, i32p, vp, vp, vp, vp, i32p, vp, sz, vp, vp, i32p, vp]
+        L.transmla_decode_step.argtypes = [pp, vp, vp, vp, i32p, i32p, vp, vp, vp, vp, vp, sz, vp, vp, i32p, vp]
         L.transmla_profile_decode_kernel.argtypes = [vp, vp]
         L.transmla_profile_decode_kernel.restype = None
         L.transmla_status_string.argtypes = [ctypes.c_int]
@@ -147,10 +147,10 @@ def transmla_decode_step_host(params, h_x, h_q_nope, h_q_pe, h_page_table, h_seq
 
 
 def transmla_decode_step(params, x, q_nope, q_pe, page_table, seqlens, w_dkv_kr, w_uk, w_uv, cache,
-                         positions_scratch, workspace, out, lse_out=None, dev_status=None, stream=None):
+                         workspace, out, lse_out=None, dev_status=None, stream=None):
     _check(lib().transmla_decode_step(
         ctypes.byref(params), _ptr(x), _ptr(q_nope), _ptr(q_pe), _ptr(page_table), _ptr(seqlens), _ptr(w_dkv_kr),
-        _ptr(w_uk), _ptr(w_uv), _ptr(cache), _ptr(positions_scratch), _ptr(workspace),
+        _ptr(w_uk), _ptr(w_uv), _ptr(cache), _ptr(workspace),
         workspace.numel() * workspace.element_size(), _ptr(out), _ptr(lse_out), _ptr(dev_status), _stream(stream)),
         'transmla_decode_step')
 

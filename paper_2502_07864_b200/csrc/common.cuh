@@ -64,9 +64,14 @@ __device__ __forceinline__ float bf16_lo(uint32_t v) { return __uint_as_float(v 
 __device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
 
 // Launchers (host).  Each enqueues on `stream` and returns the launch error, if any.
-cudaError_t launch_plan(const int32_t* seqlens, int B, int G, int32_t* cum, int32_t* plan, cudaStream_t stream);
-cudaError_t launch_absorb(const transmla_params_t& p, const __nv_bfloat16* q_nope, const __nv_bfloat16* q_pe,
-                          const __nv_bfloat16* w_uk, __nv_bfloat16* q_hat, cudaStream_t stream);
+cudaError_t launch_absorb_plan(const transmla_params_t& p, int G, const __nv_bfloat16* q_nope,
+                               const __nv_bfloat16* q_pe, const __nv_bfloat16* w_uk, __nv_bfloat16* q_hat,
+                               const int32_t* seqlens, int32_t* cum, int32_t* plan, cudaStream_t stream);
+cudaError_t launch_prologue(const transmla_params_t& p, int G, const __nv_bfloat16* x, const __nv_bfloat16* w_dkv_kr,
+                            const int32_t* page_table, __nv_bfloat16* cache, const __nv_bfloat16* q_nope,
+                            const __nv_bfloat16* q_pe, const __nv_bfloat16* w_uk, __nv_bfloat16* q_hat,
+                            const int32_t* seqlens, int32_t* cum, int32_t* plan, int32_t* dev_status,
+                            cudaStream_t stream);
 cudaError_t launch_append(const transmla_params_t& p, const __nv_bfloat16* x, const __nv_bfloat16* w,
                           const int32_t* positions, const int32_t* page_table, __nv_bfloat16* cache,
                           int32_t* dev_status, cudaStream_t stream);

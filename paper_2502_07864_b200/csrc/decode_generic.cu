@@ -266,8 +266,12 @@ static cudaError_t launch_one(const transmla_params_t& p, int G, const __nv_bflo
                               int32_t* dev_status, cudaStream_t stream) {
   using C = GenericCfg<R, DR>;
   auto kern = decode_generic_kernel<R, DR>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(C::smem_bytes));
-  if (e != cudaSuccess) return e;
+  static bool attr_set = false;  // one flag per (R, DR) instantiation
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(C::smem_bytes));
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
   const int SH = p.q_len * p.num_heads;
   dim3 grid(G, (SH + kRowBlock - 1) / kRowBlock);
   kern<<<grid, 256, C::smem_bytes, stream>>>(q_hat, cache, page_table, seqlens, cum, plan, partial_o, partial_lse,
