@@ -188,6 +188,38 @@ transmla_status_t transmla_decode_step_host(const transmla_params_t* params, con
                                             void* workspace, size_t workspace_bytes, void* h_out,
                                             float* h_lse, int32_t* h_dev_status, void* stream);
 
+/* Decode + combine without a caller workspace.  (The paper has no counterpart: this entry point
+ * exists only for the sake of how the library is deployed.)
+ *
+ * Who needs it: callers that are not in a position to allocate device memory for the workspace -
+ * an engine whose whole memory budget was handed out at start-up, code running inside another
+ * runtime's callback or capture region where an allocation would stall the device, or a host
+ * process whose device allocator belongs to a framework this library must not call into.
+ *
+ * What it does: exactly transmla_mla_decode followed by transmla_mla_combine, same arguments, same
+ * results, but the workspace is a fixed array of transmla_static_workspace_capacity() bytes (16 MiB)
+ * that is part of the library image; every GPU on which the library is loaded carries that array
+ * until the process ends.  The call allocates and frees nothing on the device.
+ *
+ * Limits and rules:
+ *   - transmla_workspace_layout(params).total_bytes must not exceed the capacity, otherwise the call
+ *     returns TRANSMLA_ERR_WORKSPACE and launches nothing.  The size grows with
+ *     (num_partitions + B - 1) * S * H * r * 4 bytes; pass a smaller params->num_partitions to fit.
+ *   - The first call on each device looks up the array's device address (with that device current)
+ *     and remembers it; make that first call outside any stream capture.
+ *   - All calls on a device share the one array and it keeps whatever the previous call left there.
+ *     A step never reads a region it has not itself written first, so no clearing is needed, but two
+ *     calls whose kernels can overlap on the GPU (different streams, no ordering) race on it: issue
+ *     them on one stream or order them with events.
+ *   q_nope, q_pe, w_uk, w_uv, cache, page_table, seqlens, out, lse_out, dev_status: device, as in
+ *   transmla_mla_decode / transmla_mla_combine. */
+size_t transmla_static_workspace_capacity(void);
+transmla_status_t transmla_mla_attention_static(const transmla_params_t* params /* host */, const void* q_nope,
+                                                const void* q_pe, const void* w_uk, const void* w_uv,
+                                                const void* cache, const int32_t* page_table,
+                                                const int32_t* seqlens, void* out, float* lse_out,
+                                                int32_t* dev_status, void* stream);
+
 /* Timing hook: the next transmla_mla_decode issued by the calling thread records `start_event`
  * immediately before and `stop_event` immediately after its split-KV kernel on that call's stream
  * (both cudaEvent_t passed as void*; NULL, NULL clears the hook).  The hook is consumed by that call. */

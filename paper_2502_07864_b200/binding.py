@@ -13,7 +13,8 @@ _LIB_PATH = os.path.join(_HERE, 'libtransmla.so')
 
 EXPORTS = ('transmla_workspace_layout', 'transmla_latent_append', 'transmla_mla_decode', 'transmla_mla_combine',
            'transmla_validate_tables', 'transmla_step_staging_bytes', 'transmla_decode_step_host',
-           'transmla_decode_step', 'transmla_profile_decode_kernel', 'transmla_status_string')
+           'transmla_decode_step', 'transmla_profile_decode_kernel', 'transmla_status_string',
+           'transmla_static_workspace_capacity', 'transmla_mla_attention_static')
 
 
 class Params(ctypes.Structure):
@@ -60,11 +61,14 @@ def lib():
         L.transmla_decode_step.argtypes = [pp, vp, vp, vp, i32p, i32p, vp, vp, vp, vp, vp, sz, vp, vp, i32p, vp]
         L.transmla_profile_decode_kernel.argtypes = [vp, vp]
         L.transmla_profile_decode_kernel.restype = None
+        L.transmla_static_workspace_capacity.argtypes = []
+        L.transmla_static_workspace_capacity.restype = sz
+        L.transmla_mla_attention_static.argtypes = [pp, vp, vp, vp, vp, vp, i32p, i32p, vp, vp, i32p, vp]
         L.transmla_status_string.argtypes = [ctypes.c_int]
         L.transmla_status_string.restype = ctypes.c_char_p
         for name in EXPORTS:
             if name not in ('transmla_step_staging_bytes', 'transmla_status_string',
-                            'transmla_profile_decode_kernel'):
+                            'transmla_profile_decode_kernel', 'transmla_static_workspace_capacity'):
                 getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -153,6 +157,18 @@ def transmla_decode_step(params, x, q_nope, q_pe, page_table, seqlens, w_dkv_kr,
         _ptr(w_uk), _ptr(w_uv), _ptr(cache), _ptr(workspace),
         workspace.numel() * workspace.element_size(), _ptr(out), _ptr(lse_out), _ptr(dev_status), _stream(stream)),
         'transmla_decode_step')
+
+
+def transmla_static_workspace_capacity():
+    return lib().transmla_static_workspace_capacity()
+
+
+def transmla_mla_attention_static(params, q_nope, q_pe, w_uk, w_uv, cache, page_table, seqlens, out, lse_out=None,
+                                  dev_status=None, stream=None):
+    """Decode + combine on the library's built-in workspace; no device buffer is created here or in the library."""
+    _check(lib().transmla_mla_attention_static(
+        ctypes.byref(params), _ptr(q_nope), _ptr(q_pe), _ptr(w_uk), _ptr(w_uv), _ptr(cache), _ptr(page_table),
+        _ptr(seqlens), _ptr(out), _ptr(lse_out), _ptr(dev_status), _stream(stream)), 'transmla_mla_attention_static')
 
 
 def transmla_profile_decode_kernel(start_event, stop_event):
