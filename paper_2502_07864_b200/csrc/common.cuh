@@ -79,6 +79,11 @@ cudaError_t launch_decode_generic(const transmla_params_t& p, int G, const __nv_
                                   const __nv_bfloat16* cache, const int32_t* page_table, const int32_t* seqlens,
                                   const int32_t* cum, const int32_t* plan, float* partial_o, float* partial_lse,
                                   int32_t* dev_status, cudaStream_t stream);
+bool decode_sm100_supported(const transmla_params_t& p);
+cudaError_t launch_decode_sm100(const transmla_params_t& p, int G, const __nv_bfloat16* q_hat,
+                                const __nv_bfloat16* cache, const int32_t* page_table, const int32_t* seqlens,
+                                const int32_t* cum, const int32_t* plan, float* partial_o, float* partial_lse,
+                                int32_t* dev_status, cudaStream_t stream);
 cudaError_t launch_combine(const transmla_params_t& p, int G, const int32_t* cum, const float* partial_o,
                            const float* partial_lse, const __nv_bfloat16* w_uv, __nv_bfloat16* out, float* lse_out,
                            cudaStream_t stream);

@@ -1,0 +1,510 @@
+// Split-KV absorbed-MLA decode (Eq. 9 right, second line) on the Blackwell tensor path:
+// TMA page loads -> shared memory -> tcgen05.mma with accumulators in tensor memory.
+//
+// Specialised for the production latent shape r = 512, dR = 64 (a cache row is 576 bf16 = 1152 B).
+// One CTA = one (partition, block of 32 query rows); it walks its segments page by page.
+//
+// Tile plan per 64-token page
+//   S  [128 x 64]   = Q_hat (tensor memory, the 32 rows replicated into the four 32-lane quadrants)
+//                     x K_hat^T (the page in shared memory, K-major, 128-byte swizzle), K = 576
+//   O^T[512 x 32]  += C^T (the same shared-memory page read MN-major, four 128-row tiles)
+//                     x P^T (32 rows x 64 tokens, bf16, shared memory, K-major)
+// O is kept transposed (latent index on the tensor-memory lanes, query rows on the columns) so that
+// the accumulator costs 4 x 32 columns instead of 512, which leaves room for Q_hat (288 columns) and
+// S (64 columns) in the 512-column tensor memory, and so that no padded query row costs PV work.
+//
+// Warp roles: warps 0-3 softmax + epilogue (warp w owns tensor-memory lanes 32w..32w+31, i.e. replica w
+// of the 32 query rows, and the probabilities of tokens 16w..16w+15 of every page); warp 4 lane 0
+// issues TMA; warp 5 lane 0 issues MMA.  All waits are bounded: on expiry the CTA raises
+// TRANSMLA_DEV_TIMEOUT, every later wait returns at once, and control flow stays identical, so the CTA
+// still reaches its teardown and frees its tensor memory.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+
+#include <mutex>
+
+#include "common.cuh"
+
+namespace transmla {
+namespace sm100 {
+
+constexpr int R = 512, DR = 64, K = R + DR;
+constexpr int kChunks = K / 64;                       // 9 sub-tiles of 64 columns (128 bytes) per page
+constexpr int kSubTileBytes = kPage * 128;            // 8192
+constexpr int kStageBytes = kChunks * kSubTileBytes;  // 73728
+constexpr int kStages = 3;
+constexpr int kPBytes = kRowBlock * 128;              // 4096: P[32 rows][64 tokens] bf16
+constexpr int kThreads = 192;
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kColQ = 0, kColS = 288, kColO = 352;  // tensor-memory column map: Q_hat, S, O^T (4 x 32)
+
+// shared-memory map (offsets from a 1024-byte aligned base)
+constexpr int kOffStage = 0;
+constexpr int kOffP = kStages * kStageBytes;      // 2 buffers
+constexpr int kOffBar = kOffP + 2 * kPBytes;      // mbarriers (8 bytes each)
+constexpr int kNumBars = 2 * kStages + 6;
+constexpr int kOffMisc = kOffBar + 128;
+// misc: m_s[2][32] f32, alpha_s[2][32] f32, flag_s[2] i32, l_part[4][32] f32, inv_l[32] f32, tmem base, abort
+constexpr int kMiscBytes = 256 + 256 + 16 + 512 + 128 + 16;
+constexpr int kSmemBytes = kOffMisc + kMiscBytes + 1024;  // + slack for the 1024-byte alignment
+static_assert(kSmemBytes <= 232448, "shared memory budget");
+
+enum { BAR_KV_FULL = 0, BAR_KV_EMPTY = kStages, BAR_Q_READY = 2 * kStages, BAR_S_FULL, BAR_S_FREE, BAR_P_READY,
+       BAR_PV_DONE0, BAR_PV_DONE1 };
+
+constexpr long long kWaitCycles = 400000000LL;  // ~0.2 s at 2 GHz
+
+// ---------------------------------------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns at once when the CTA has already given up.
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* dev_status) {
+  if (*abort_flag) return;
+  if (mbar_try_wait(bar, parity)) return;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (*abort_flag) return;
+    if (clock64() - t0 > kWaitCycles) {
+      *abort_flag = 1;
+      set_status(dev_status, TRANSMLA_DEV_TIMEOUT);
+      return;
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem desc]
+__device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
+      ::"r"(d), "r"(a), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// D[tmem] (+)= A[smem desc] * B[smem desc]
+__device__ __forceinline__ void mma_ss(uint32_t d, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+#define TM_R4(v, i) "=r"(v[i]), "=r"(v[i + 1]), "=r"(v[i + 2]), "=r"(v[i + 3])
+#define TM_R16(v, i) TM_R4(v, i), TM_R4(v, i + 4), TM_R4(v, i + 8), TM_R4(v, i + 12)
+#define TM_W4(v, i) "r"(v[i]), "r"(v[i + 1]), "r"(v[i + 2]), "r"(v[i + 3])
+#define TM_W16(v, i) TM_W4(v, i), TM_W4(v, i + 4), TM_W4(v, i + 8), TM_W4(v, i + 12)
+
+// 32 lanes x 16 consecutive 32-bit columns: thread i of the warp gets lane (base lane + i).
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* v) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : TM_R16(v, 0)
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* v) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : TM_R16(v, 0), TM_R16(v, 16)
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};"
+      ::TM_W16(v, 0), "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31};"
+      ::TM_W16(v, 0), TM_W16(v, 16), "r"(taddr)
+      : "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle: start address, leading and stride byte offsets
+// (all in 16-byte units), descriptor version 1, layout type 2.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return static_cast<uint64_t>((addr & 0x3FFFFu) >> 4) | (static_cast<uint64_t>(lbo_bytes >> 4) << 16) |
+         (static_cast<uint64_t>(sbo_bytes >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor of kind::f16: fp32 accumulator, bf16 A and B, M = 128.
+__host__ __device__ constexpr uint32_t instr_desc(int n, bool a_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | (static_cast<uint32_t>(n >> 3) << 17) |
+         (static_cast<uint32_t>(128 >> 4) << 24);
+}
+
+// ---------------------------------------------------------------------------------------------- kernel
+__global__ void __launch_bounds__(kThreads, 1)
+decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __nv_bfloat16* __restrict__ q_hat,
+                    const int32_t* __restrict__ page_table, const int32_t* __restrict__ seqlens,
+                    const int32_t* __restrict__ cum, const int32_t* __restrict__ plan, float* __restrict__ partial_o,
+                    float* __restrict__ partial_lse, int32_t* dev_status, int S, int H, int num_pages, int max_pages,
+                    float scale_log2) {
+  extern __shared__ unsigned char smem_unaligned[];
+  const uint32_t raw = smem_u32(smem_unaligned);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  unsigned char* sm = smem_unaligned + (base - raw);
+  float* m_s = reinterpret_cast<float*>(sm + kOffMisc);            // [2][32]
+  float* alpha_s = m_s + 64;                                       // [2][32]
+  int* flag_s = reinterpret_cast<int*>(alpha_s + 64);              // [2] (+2 pad)
+  float* l_part = reinterpret_cast<float*>(flag_s + 4);            // [4][32]
+  float* inv_l = l_part + 128;                                     // [32]
+  uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(inv_l + 32);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_base_s + 1);
+  auto bar = [&](int i) -> uint32_t { return base + kOffBar + 8 * i; };
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int part = blockIdx.x, rb = blockIdx.y;
+  const int SH = S * H;
+  const int4 pl = reinterpret_cast<const int4*>(plan)[part];
+
+  if (tid == 0) {
+    for (int i = 0; i < kStages; ++i) { mbar_init(bar(BAR_KV_FULL + i), 1); mbar_init(bar(BAR_KV_EMPTY + i), 1); }
+    mbar_init(bar(BAR_Q_READY), 128);
+    mbar_init(bar(BAR_S_FULL), 1);
+    mbar_init(bar(BAR_S_FREE), 128);
+    mbar_init(bar(BAR_P_READY), 128);
+    mbar_init(bar(BAR_PV_DONE0), 1);
+    mbar_init(bar(BAR_PV_DONE1), 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_base_s)), "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_base_s;
+
+  if (pl.y > pl.x) {
+    if (warp == 4) {
+      // ======================================================================== TMA producer
+      if (lane == 0) {
+        int g = 0;  // pages issued by this CTA so far
+        for (int b = pl.z; b <= pl.w; ++b) {
+          const int c0 = cum[b];
+          const int pg_lo = max(pl.x, c0) - c0, pg_hi = min(pl.y, cum[b + 1]) - c0;
+          for (int pj = pg_lo; pj < pg_hi; ++pj, ++g) {
+            const int stage = g % kStages, use = g / kStages;
+            int idx = page_table[static_cast<size_t>(b) * max_pages + pj];
+            if (idx < 0 || idx >= num_pages) { set_status(dev_status, TRANSMLA_DEV_BAD_PAGE); idx = 0; }
+            mbar_wait(bar(BAR_KV_EMPTY + stage), (use & 1) ^ 1, abort_flag, dev_status);
+            if (*abort_flag) continue;
+            mbar_arrive_expect_tx(bar(BAR_KV_FULL + stage), kStageBytes);
+            const uint32_t dst = base + kOffStage + stage * kStageBytes;
+#pragma unroll
+            for (int c = 0; c < kChunks; ++c)
+              tma_load_2d(dst + c * kSubTileBytes, &cache_map, c * 64, idx * kPage, bar(BAR_KV_FULL + stage));
+          }
+        }
+      }
+    } else if (warp == 5) {
+      // ======================================================================== MMA issuer
+      if (lane == 0) {
+        constexpr uint32_t idesc_qk = instr_desc(kPage, false);
+        constexpr uint32_t idesc_pv = instr_desc(kRowBlock, true);
+        int g = 0, seg = 0;
+        auto issue_pv = [&](int gp, bool first_of_segment) {  // O^T += C^T P^T for CTA page gp
+          const int stage = gp % kStages;
+          mbar_wait(bar(BAR_P_READY), gp & 1, abort_flag, dev_status);
+          tc_fence_after();
+          const uint32_t pg = base + kOffStage + stage * kStageBytes;
+          const uint32_t pb = base + kOffP + (gp & 1) * kPBytes;
+#pragma unroll
+          for (int t = 0; t < 4; ++t) {
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+              const uint64_t a_desc = smem_desc(pg + (2 * t) * kSubTileBytes + kk * 2048, kSubTileBytes, 1024);
+              const uint64_t b_desc = smem_desc(pb + kk * 32, 16, 1024);
+              mma_ss(tmem + kColO + t * 32, a_desc, b_desc, idesc_pv, (first_of_segment && kk == 0) ? 0u : 1u);
+            }
+          }
+          tc_commit(bar(BAR_KV_EMPTY + stage));
+          tc_commit(bar(BAR_PV_DONE0 + (gp & 1)));
+        };
+        for (int b = pl.z; b <= pl.w; ++b) {
+          const int c0 = cum[b];
+          const int pg_lo = max(pl.x, c0) - c0, pg_hi = min(pl.y, cum[b + 1]) - c0;
+          if (pg_hi <= pg_lo) continue;
+          mbar_wait(bar(BAR_Q_READY), seg & 1, abort_flag, dev_status);
+          ++seg;
+          for (int pj = pg_lo; pj < pg_hi; ++pj, ++g) {
+            const int stage = g % kStages, use = g / kStages;
+            mbar_wait(bar(BAR_KV_FULL + stage), use & 1, abort_flag, dev_status);
+            if (g > 0) mbar_wait(bar(BAR_S_FREE), (g - 1) & 1, abort_flag, dev_status);
+            tc_fence_after();
+            const uint32_t pg = base + kOffStage + stage * kStageBytes;
+#pragma unroll
+            for (int c = 0; c < kChunks; ++c) {
+#pragma unroll
+              for (int kk = 0; kk < 4; ++kk) {
+                const uint64_t b_desc = smem_desc(pg + c * kSubTileBytes + kk * 32, 16, 1024);
+                mma_ts(tmem + kColS, tmem + kColQ + c * 32 + kk * 8, b_desc, idesc_qk, (c | kk) ? 1u : 0u);
+              }
+            }
+            tc_commit(bar(BAR_S_FULL));
+            if (pj > pg_lo) issue_pv(g - 1, pj - 1 == pg_lo);
+          }
+          issue_pv(g - 1, pg_hi - 1 == pg_lo);
+        }
+      }
+    } else {
+      // ======================================================================== softmax + epilogue (warps 0-3)
+      const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
+      const int my_row = rb * kRowBlock + lane;  // query row of this thread (same in all four replicas)
+      int g = 0, seg = 0;
+      for (int b = pl.z; b <= pl.w; ++b) {
+        const int c0 = cum[b];
+        const int pg_lo = max(pl.x, c0) - c0, pg_hi = min(pl.y, cum[b + 1]) - c0;
+        if (pg_hi <= pg_lo) continue;
+        const int L = seqlens[b];
+        const int slot = part + b;
+        const int n_vis = my_row < SH ? L - (S - 1 - my_row / H) : 0;
+
+        // ---- Q_hat rows -> tensor memory (this warp's replica), 32 columns (64 elements) at a time
+        {
+          const uint4* src = reinterpret_cast<const uint4*>(q_hat + (static_cast<size_t>(b) * SH + min(my_row, SH - 1)) * K);
+          for (int c = 0; c < K / 64; ++c) {
+            uint32_t v[32];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              uint4 x = make_uint4(0, 0, 0, 0);
+              if (my_row < SH) x = src[c * 8 + j];
+              v[4 * j] = x.x; v[4 * j + 1] = x.y; v[4 * j + 2] = x.z; v[4 * j + 3] = x.w;
+            }
+            tmem_st32(tmem + lane_base + kColQ + c * 32, v);
+          }
+          tc_wait_st();
+          tc_fence_before();
+          mbar_arrive(bar(BAR_Q_READY));
+          ++seg;
+        }
+
+        float m_used = -INFINITY, l_run = 0.f;
+        for (int pj = pg_lo; pj < pg_hi; ++pj, ++g) {
+          const int stage = g % kStages;
+          const int idx = page_table[static_cast<size_t>(b) * max_pages + pj];
+          const bool page_ok = idx >= 0 && idx < num_pages;
+          const int tok_end = page_ok ? n_vis - pj * kPage : 0;           // tokens [0, tok_end) of the page are visible
+          const int valid = page_ok ? min(kPage, L - pj * kPage) : 0;      // rows [valid, 64) must read as zero
+          const bool first = pj == pg_lo;
+          const int buf = g & 1;
+
+          mbar_wait(bar(BAR_S_FULL), g & 1, abort_flag, dev_status);
+          tc_fence_after();
+          uint32_t sq[16];  // this warp's 16 tokens of its row
+          float rowmax = -INFINITY;
+          if (warp == 0) {
+            uint32_t sv[64];
+            tmem_ld32(tmem + lane_base + kColS, sv);
+            tmem_ld32(tmem + lane_base + kColS + 32, sv + 32);
+            tc_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 64; ++j)
+              rowmax = fmaxf(rowmax, j < tok_end ? __uint_as_float(sv[j]) * scale_log2 : -INFINITY);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) sq[j] = sv[j];
+          } else {
+            tmem_ld16(tmem + lane_base + kColS + warp * 16, sq);
+            tc_wait_ld();
+          }
+          tc_fence_before();
+          mbar_arrive(bar(BAR_S_FREE));
+
+          if (warp == 0) {
+            // Lazy rescale: the reference maximum only moves when some row's new maximum exceeds it by 2^8.
+            float alpha = 1.f;
+            bool need = false;
+            if (first) {
+              m_used = rowmax;
+            } else {
+              need = rowmax > m_used + 8.f;
+            }
+            const bool any = __any_sync(0xffffffffu, need);
+            if (any) {
+              const float m_new = fmaxf(m_used, rowmax);
+              alpha = (m_new == -INFINITY) ? 1.f : exp2f(m_used - m_new);
+              m_used = m_new;
+            }
+            m_s[buf * 32 + lane] = m_used;
+            alpha_s[buf * 32 + lane] = alpha;
+            if (lane == 0) flag_s[buf] = any ? 1 : 0;
+          }
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+          const float m_ref = m_s[buf * 32 + lane];
+          const bool rescale = flag_s[buf] != 0;
+          if (rescale) l_run *= alpha_s[buf * 32 + lane];
+          m_used = m_ref;
+
+          // ---- probabilities of tokens 16*warp .. 16*warp+15
+          uint32_t pk[8];
+          float psum = 0.f;
+#pragma unroll
+          for (int j = 0; j < 16; j += 2) {
+            const int t0 = warp * 16 + j;
+            const float p0 = t0 < tok_end ? exp2f(__uint_as_float(sq[j]) * scale_log2 - m_ref) : 0.f;
+            const float p1 = t0 + 1 < tok_end ? exp2f(__uint_as_float(sq[j + 1]) * scale_log2 - m_ref) : 0.f;
+            psum += p0 + p1;
+            pk[j >> 1] = pack_bf16(p0, p1);
+          }
+          l_run += psum;
+
+          // ---- P buffer `buf` is free once PV of CTA page g-2 is done
+          if (g >= 2) mbar_wait(bar(BAR_PV_DONE0 + buf), ((g >> 1) - 1) & 1, abort_flag, dev_status);
+          {
+            unsigned char* prow = sm + kOffP + buf * kPBytes + lane * 128;
+            const int c0w = 2 * warp, sw = lane & 7;
+            *reinterpret_cast<uint4*>(prow + ((c0w ^ sw) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            *reinterpret_cast<uint4*>(prow + (((c0w + 1) ^ sw) << 4)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+          }
+          // ---- rows of the page beyond the sequence must contribute exact zeros to O
+          if (valid < kPage) {
+            unsigned char* pgp = sm + kOffStage + stage * kStageBytes;
+            const int rows = kPage - valid;
+            for (int i = tid; i < rows * 8 * 8; i += 128) {  // rows x 8 latent sub-tiles x 8 chunks of 16 bytes
+              const int rr = valid + i / 64, t = (i >> 3) & 7, ch = i & 7;
+              *reinterpret_cast<uint4*>(pgp + t * kSubTileBytes + rr * 128 + ch * 16) = make_uint4(0, 0, 0, 0);
+            }
+          }
+          // ---- rescale O^T by alpha (columns = query rows) once the previous PV has landed
+          if (rescale) {
+            if (g >= 1) mbar_wait(bar(BAR_PV_DONE0 + ((g - 1) & 1)), ((g - 1) >> 1) & 1, abort_flag, dev_status);
+            tc_fence_after();
+#pragma unroll 1
+            for (int t = 0; t < 4; ++t) {
+              uint32_t ov[32];
+              tmem_ld32(tmem + lane_base + kColO + t * 32, ov);
+              tc_wait_ld();
+#pragma unroll
+              for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * alpha_s[buf * 32 + j]);
+              tmem_st32(tmem + lane_base + kColO + t * 32, ov);
+            }
+            tc_wait_st();
+          }
+          fence_proxy_async();
+          tc_fence_before();
+          mbar_arrive(bar(BAR_P_READY));
+        }
+
+        // ---- epilogue of the segment: wait for the last PV, normalise, store O (transposed back) and lse
+        l_part[warp * 32 + lane] = l_run;
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        const float l_tot = l_part[lane] + l_part[32 + lane] + l_part[64 + lane] + l_part[96 + lane];
+        if (warp == 0) {
+          inv_l[lane] = l_tot > 0.f ? 1.f / l_tot : 0.f;
+          if (my_row < SH)
+            partial_lse[static_cast<size_t>(slot) * SH + my_row] = l_tot > 0.f ? (m_used + log2f(l_tot)) * kLn2 : -INFINITY;
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        const int g_last = g - 1;
+        mbar_wait(bar(BAR_PV_DONE0 + (g_last & 1)), (g_last >> 1) & 1, abort_flag, dev_status);
+        tc_fence_after();
+        float* dst = partial_o + (static_cast<size_t>(slot) * SH + rb * kRowBlock) * R + warp * 32 + lane;
+#pragma unroll 1
+        for (int t = 0; t < 4; ++t) {
+          uint32_t ov[32];
+          tmem_ld32(tmem + lane_base + kColO + t * 32, ov);
+          tc_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (rb * kRowBlock + j < SH) dst[static_cast<size_t>(j) * R + t * 128] = __uint_as_float(ov[j]) * inv_l[j];
+        }
+        tc_fence_before();
+        asm volatile("bar.sync 1, 128;" ::: "memory");  // inv_l / l_part are reused by the next segment
+      }
+    }
+  }
+
+  // ---- teardown: everyone arrives, tensor memory is returned
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 0) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------------------------------------- host
+static PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
+  static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(p);
+  });
+  return fn;
+}
+
+}  // namespace sm100
+
+bool decode_sm100_supported(const transmla_params_t& p) { return p.kv_lora_rank == sm100::R && p.qk_rope_dim == sm100::DR; }
+
+cudaError_t launch_decode_sm100(const transmla_params_t& p, int G, const __nv_bfloat16* q_hat,
+                                const __nv_bfloat16* cache, const int32_t* page_table, const int32_t* seqlens,
+                                const int32_t* cum, const int32_t* plan, float* partial_o, float* partial_lse,
+                                int32_t* dev_status, cudaStream_t stream) {
+  using namespace sm100;
+  auto encode = encode_fn();
+  if (encode == nullptr) return cudaErrorNotSupported;
+  // The pool as a 2-D tensor [num_pages * 64 rows, 576 columns]; one box = 64 rows x 64 columns (128 bytes),
+  // written to shared memory with the 128-byte swizzle the MMA descriptors expect.
+  CUtensorMap map;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(K), static_cast<cuuint64_t>(p.num_pages) * kPage};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(K) * sizeof(__nv_bfloat16)};
+  const cuuint32_t box[2] = {64, kPage};
+  const cuuint32_t elem_strides[2] = {1, 1};
+  if (encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(cache), dims, strides, box, elem_strides,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return cudaErrorInvalidValue;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(decode_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  const int SH = p.q_len * p.num_heads;
+  dim3 grid(G, (SH + kRowBlock - 1) / kRowBlock);
+  decode_sm100_kernel<<<grid, kThreads, kSmemBytes, stream>>>(map, q_hat, page_table, seqlens, cum, plan, partial_o,
+                                                              partial_lse, dev_status, p.q_len, p.num_heads, p.num_pages,
+                                                              p.max_pages_per_seq, p.softmax_scale * kLog2e);
+  return cudaGetLastError();
+}
+
+}  // namespace transmla
