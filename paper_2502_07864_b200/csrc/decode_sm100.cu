@@ -15,7 +15,7 @@
 //
 // Warp roles: warps 0-3 softmax + epilogue (warp w owns tensor-memory lanes 32w..32w+31, i.e. replica w
 // of the 32 query rows, and the probabilities of tokens 16w..16w+15 of every page); warp 4 lane 0
-// issues TMA; warp 5 lane 0 issues MMA.  All waits are bounded: on expiry the CTA raises
+// issues TMA; warp 5 issues MMA (warp-uniform control flow, one elected lane per instruction).  All waits are bounded: on expiry the CTA raises
 // TRANSMLA_DEV_TIMEOUT, every later wait returns at once, and control flow stays identical, so the CTA
 // still reaches its teardown and frees its tensor memory.
 #include <cuda.h>
@@ -87,6 +87,13 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
   }
 }
+// True in exactly one lane of a converged warp.  Code around it stays warp-uniform, so descriptors and
+// addresses can live in uniform registers instead of being moved there for every instruction.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n.reg .pred p;\nelect.sync _|p, 0xffffffff;\nselp.u32 %0, 1, 0, p;\n}" : "=r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
@@ -157,6 +164,9 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
   return static_cast<uint64_t>((addr & 0x3FFFFu) >> 4) | (static_cast<uint64_t>(lbo_bytes >> 4) << 16) |
          (static_cast<uint64_t>(sbo_bytes >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
+// The same descriptor `bytes` further on (bytes is a multiple of 16; the tile stays inside the 256 KB window,
+// so the 14-bit address field cannot carry).
+__device__ __forceinline__ uint64_t desc_advance(uint64_t desc, uint32_t bytes) { return desc + (bytes >> 4); }
 // Instruction descriptor of kind::f16: fp32 accumulator, bf16 A and B, M = 128.
 __host__ __device__ constexpr uint32_t instr_desc(int n, bool a_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | (static_cast<uint32_t>(n >> 3) << 17) |
@@ -233,7 +243,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __nv_bf
       }
     } else if (warp == 5) {
       // ======================================================================== MMA issuer
-      if (lane == 0) {
+      {
         constexpr uint32_t idesc_qk = instr_desc(kPage, false);
         constexpr uint32_t idesc_pv = instr_desc(kRowBlock, true);
         int g = 0, seg = 0;
@@ -241,19 +251,23 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __nv_bf
           const int stage = gp % kStages;
           mbar_wait(bar(BAR_P_READY), gp & 1, abort_flag, dev_status);
           tc_fence_after();
-          const uint32_t pg = base + kOffStage + stage * kStageBytes;
-          const uint32_t pb = base + kOffP + (gp & 1) * kPBytes;
+          const uint64_t a0 = smem_desc(base + kOffStage + stage * kStageBytes, kSubTileBytes, 1024);
+          const uint64_t b0 = smem_desc(base + kOffP + (gp & 1) * kPBytes, 16, 1024);
+          const uint32_t acc0 = first_of_segment ? 0u : 1u;
 #pragma unroll
-          for (int t = 0; t < 4; ++t) {
+          for (int kk = 0; kk < 4; ++kk) {
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
-              const uint64_t a_desc = smem_desc(pg + (2 * t) * kSubTileBytes + kk * 2048, kSubTileBytes, 1024);
-              const uint64_t b_desc = smem_desc(pb + kk * 32, 16, 1024);
-              mma_ss(tmem + kColO + t * 32, a_desc, b_desc, idesc_pv, (first_of_segment && kk == 0) ? 0u : 1u);
+            for (int t = 0; t < 4; ++t) {
+              if (elect_one())
+                mma_ss(tmem + kColO + t * 32, desc_advance(a0, (2 * t) * kSubTileBytes + kk * 2048),
+                       desc_advance(b0, kk * 32), idesc_pv, kk == 0 ? acc0 : 1u);
             }
           }
-          tc_commit(bar(BAR_KV_EMPTY + stage));
-          tc_commit(bar(BAR_PV_DONE0 + (gp & 1)));
+          if (elect_one()) {
+            tc_commit(bar(BAR_KV_EMPTY + stage));
+            tc_commit(bar(BAR_PV_DONE0 + (gp & 1)));
+          }
+          __syncwarp();
         };
         for (int b = pl.z; b <= pl.w; ++b) {
           const int c0 = cum[b];
@@ -266,16 +280,18 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __nv_bf
             mbar_wait(bar(BAR_KV_FULL + stage), use & 1, abort_flag, dev_status);
             if (g > 0) mbar_wait(bar(BAR_S_FREE), (g - 1) & 1, abort_flag, dev_status);
             tc_fence_after();
-            const uint32_t pg = base + kOffStage + stage * kStageBytes;
+            const uint64_t k0 = smem_desc(base + kOffStage + stage * kStageBytes, 16, 1024);
 #pragma unroll
             for (int c = 0; c < kChunks; ++c) {
 #pragma unroll
               for (int kk = 0; kk < 4; ++kk) {
-                const uint64_t b_desc = smem_desc(pg + c * kSubTileBytes + kk * 32, 16, 1024);
-                mma_ts(tmem + kColS, tmem + kColQ + c * 32 + kk * 8, b_desc, idesc_qk, (c | kk) ? 1u : 0u);
+                if (elect_one())
+                  mma_ts(tmem + kColS, tmem + kColQ + c * 32 + kk * 8, desc_advance(k0, c * kSubTileBytes + kk * 32),
+                         idesc_qk, (c | kk) ? 1u : 0u);
               }
             }
-            tc_commit(bar(BAR_S_FULL));
+            if (elect_one()) tc_commit(bar(BAR_S_FULL));
+            __syncwarp();
             if (pj > pg_lo) issue_pv(g - 1, pj - 1 == pg_lo);
           }
           issue_pv(g - 1, pg_hi - 1 == pg_lo);
