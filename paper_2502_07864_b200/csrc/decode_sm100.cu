@@ -34,6 +34,7 @@ constexpr int kSubTileBytes = kPage * 128;            // 8192
 constexpr int kStageBytes = kChunks * kSubTileBytes;  // 73728
 constexpr int kStages = 3;
 constexpr int kPBytes = kRowBlock * 128;              // 4096: P[32 rows][64 tokens] bf16
+constexpr int kQTileBytes = kRowBlock * 128;          // 4096: one 64-column sub-tile of the 32 query rows
 constexpr int kThreads = 192;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColQ = 0, kColS = 288, kColO = 352;  // tensor-memory column map: Q_hat, S, O^T (4 x 32)
@@ -42,7 +43,6 @@ constexpr uint32_t kColQ = 0, kColS = 288, kColO = 352;  // tensor-memory column
 constexpr int kOffStage = 0;
 constexpr int kOffP = kStages * kStageBytes;      // 2 buffers
 constexpr int kOffBar = kOffP + 2 * kPBytes;      // mbarriers (8 bytes each)
-constexpr int kNumBars = 2 * kStages + 6;
 constexpr int kOffMisc = kOffBar + 128;
 // misc: m_s[2][32] f32, alpha_s[2][32] f32, flag_s[2] i32, l_part[4][32] f32, inv_l[32] f32, tmem base, abort
 constexpr int kMiscBytes = 256 + 256 + 16 + 512 + 128 + 16;
@@ -175,7 +175,7 @@ __host__ __device__ constexpr uint32_t instr_desc(int n, bool a_mn_major) {
 
 // ---------------------------------------------------------------------------------------------- kernel
 __global__ void __launch_bounds__(kThreads, 1)
-decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __nv_bfloat16* __restrict__ q_hat,
+decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_constant__ CUtensorMap q_map,
                     const int32_t* __restrict__ page_table, const int32_t* __restrict__ seqlens,
                     const int32_t* __restrict__ cum, const int32_t* __restrict__ plan, float* __restrict__ partial_o,
                     float* __restrict__ partial_lse, int32_t* dev_status, int S, int H, int num_pages, int max_pages,
@@ -222,23 +222,41 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __nv_bf
   if (pl.y > pl.x) {
     if (warp == 4) {
       // ======================================================================== TMA producer
-      if (lane == 0) {
-        int g = 0;  // pages issued by this CTA so far
-        for (int b = pl.z; b <= pl.w; ++b) {
-          const int c0 = cum[b];
-          const int pg_lo = max(pl.x, c0) - c0, pg_hi = min(pl.y, cum[b + 1]) - c0;
-          for (int pj = pg_lo; pj < pg_hi; ++pj, ++g) {
-            const int stage = g % kStages, use = g / kStages;
-            int idx = page_table[static_cast<size_t>(b) * max_pages + pj];
-            if (idx < 0 || idx >= num_pages) { set_status(dev_status, TRANSMLA_DEV_BAD_PAGE); idx = 0; }
-            mbar_wait(bar(BAR_KV_EMPTY + stage), (use & 1) ^ 1, abort_flag, dev_status);
-            if (*abort_flag) continue;
+      // The ring carries, per segment, one item with the 32 absorbed query rows followed by the segment's pages.
+      int g = 0;  // ring items issued by this CTA so far
+      auto acquire = [&](int gi) -> uint32_t {  // waits for the stage of ring item gi; returns its index
+        const int stage = gi % kStages, use = gi / kStages;
+        mbar_wait(bar(BAR_KV_EMPTY + stage), (use & 1) ^ 1, abort_flag, dev_status);
+        return stage;
+      };
+      for (int b = pl.z; b <= pl.w; ++b) {
+        const int c0 = cum[b];
+        const int pg_lo = max(pl.x, c0) - c0, pg_hi = min(pl.y, cum[b + 1]) - c0;
+        if (pg_hi <= pg_lo) continue;
+        {
+          const uint32_t stage = acquire(g);
+          if (!*abort_flag && elect_one()) {
+            mbar_arrive_expect_tx(bar(BAR_KV_FULL + stage), kChunks * kQTileBytes);
+            const uint32_t dst = base + kOffStage + stage * kStageBytes;
+#pragma unroll
+            for (int c = 0; c < kChunks; ++c)
+              tma_load_2d(dst + c * kQTileBytes, &q_map, c * 64, b * SH + rb * kRowBlock, bar(BAR_KV_FULL + stage));
+          }
+          __syncwarp();
+          ++g;
+        }
+        for (int pj = pg_lo; pj < pg_hi; ++pj, ++g) {
+          int idx = page_table[static_cast<size_t>(b) * max_pages + pj];
+          if (idx < 0 || idx >= num_pages) { if (lane == 0) set_status(dev_status, TRANSMLA_DEV_BAD_PAGE); idx = 0; }
+          const uint32_t stage = acquire(g);
+          if (!*abort_flag && elect_one()) {
             mbar_arrive_expect_tx(bar(BAR_KV_FULL + stage), kStageBytes);
             const uint32_t dst = base + kOffStage + stage * kStageBytes;
 #pragma unroll
             for (int c = 0; c < kChunks; ++c)
               tma_load_2d(dst + c * kSubTileBytes, &cache_map, c * 64, idx * kPage, bar(BAR_KV_FULL + stage));
           }
+          __syncwarp();
         }
       }
     } else if (warp == 5) {
@@ -246,9 +264,9 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __nv_bf
       {
         constexpr uint32_t idesc_qk = instr_desc(kPage, false);
         constexpr uint32_t idesc_pv = instr_desc(kRowBlock, true);
-        int g = 0, seg = 0;
-        auto issue_pv = [&](int gp, bool first_of_segment) {  // O^T += C^T P^T for CTA page gp
-          const int stage = gp % kStages;
+        int g = 0, n = 0, seg = 0;  // ring items, pages, segments handled so far
+        auto issue_pv = [&](int gr, int gp, bool first_of_segment) {  // O^T += C^T P^T for page gp held in ring item gr
+          const int stage = gr % kStages;
           mbar_wait(bar(BAR_P_READY), gp & 1, abort_flag, dev_status);
           tc_fence_after();
           const uint64_t a0 = smem_desc(base + kOffStage + stage * kStageBytes, kSubTileBytes, 1024);
@@ -273,12 +291,13 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __nv_bf
           const int c0 = cum[b];
           const int pg_lo = max(pl.x, c0) - c0, pg_hi = min(pl.y, cum[b + 1]) - c0;
           if (pg_hi <= pg_lo) continue;
+          ++g;  // the segment's query item is consumed by the softmax warps
           mbar_wait(bar(BAR_Q_READY), seg & 1, abort_flag, dev_status);
           ++seg;
-          for (int pj = pg_lo; pj < pg_hi; ++pj, ++g) {
+          for (int pj = pg_lo; pj < pg_hi; ++pj, ++g, ++n) {
             const int stage = g % kStages, use = g / kStages;
             mbar_wait(bar(BAR_KV_FULL + stage), use & 1, abort_flag, dev_status);
-            if (g > 0) mbar_wait(bar(BAR_S_FREE), (g - 1) & 1, abort_flag, dev_status);
+            if (n > 0) mbar_wait(bar(BAR_S_FREE), (n - 1) & 1, abort_flag, dev_status);
             tc_fence_after();
             const uint64_t k0 = smem_desc(base + kOffStage + stage * kStageBytes, 16, 1024);
 #pragma unroll
@@ -292,16 +311,16 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __nv_bf
             }
             if (elect_one()) tc_commit(bar(BAR_S_FULL));
             __syncwarp();
-            if (pj > pg_lo) issue_pv(g - 1, pj - 1 == pg_lo);
+            if (pj > pg_lo) issue_pv(g - 1, n - 1, pj - 1 == pg_lo);
           }
-          issue_pv(g - 1, pg_hi - 1 == pg_lo);
+          issue_pv(g - 1, n - 1, pg_hi - 1 == pg_lo);
         }
       }
     } else {
       // ======================================================================== softmax + epilogue (warps 0-3)
       const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
       const int my_row = rb * kRowBlock + lane;  // query row of this thread (same in all four replicas)
-      int g = 0, seg = 0;
+      int g = 0, n = 0;  // ring items and pages handled so far
       for (int b = pl.z; b <= pl.w; ++b) {
         const int c0 = cum[b];
         const int pg_lo = max(pl.x, c0) - c0, pg_hi = min(pl.y, cum[b + 1]) - c0;
@@ -310,15 +329,18 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __nv_bf
         const int slot = part + b;
         const int n_vis = my_row < SH ? L - (S - 1 - my_row / H) : 0;
 
-        // ---- Q_hat rows -> tensor memory (this warp's replica), 32 columns (64 elements) at a time
+        // ---- Q_hat rows: shared memory (swizzled sub-tiles of 32 rows x 128 bytes) -> this warp's replica in
+        //      tensor memory, 32 columns (64 elements) at a time; then the ring stage is handed back
         {
-          const uint4* src = reinterpret_cast<const uint4*>(q_hat + (static_cast<size_t>(b) * SH + min(my_row, SH - 1)) * K);
-          for (int c = 0; c < K / 64; ++c) {
+          const int stage = g % kStages, use = g / kStages;
+          mbar_wait(bar(BAR_KV_FULL + stage), use & 1, abort_flag, dev_status);
+          const unsigned char* qrow = sm + kOffStage + stage * kStageBytes + lane * 128;
+#pragma unroll 1
+          for (int c = 0; c < kChunks; ++c) {
             uint32_t v[32];
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-              uint4 x = make_uint4(0, 0, 0, 0);
-              if (my_row < SH) x = src[c * 8 + j];
+              const uint4 x = *reinterpret_cast<const uint4*>(qrow + c * kQTileBytes + ((j ^ (lane & 7)) << 4));
               v[4 * j] = x.x; v[4 * j + 1] = x.y; v[4 * j + 2] = x.z; v[4 * j + 3] = x.w;
             }
             tmem_st32(tmem + lane_base + kColQ + c * 32, v);
@@ -326,20 +348,22 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __nv_bf
           tc_wait_st();
           tc_fence_before();
           mbar_arrive(bar(BAR_Q_READY));
-          ++seg;
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+          if (tid == 0) mbar_arrive(bar(BAR_KV_EMPTY + stage));
+          ++g;
         }
 
         float m_used = -INFINITY, l_run = 0.f;
-        for (int pj = pg_lo; pj < pg_hi; ++pj, ++g) {
+        for (int pj = pg_lo; pj < pg_hi; ++pj, ++g, ++n) {
           const int stage = g % kStages;
           const int idx = page_table[static_cast<size_t>(b) * max_pages + pj];
           const bool page_ok = idx >= 0 && idx < num_pages;
           const int tok_end = page_ok ? n_vis - pj * kPage : 0;           // tokens [0, tok_end) of the page are visible
           const int valid = page_ok ? min(kPage, L - pj * kPage) : 0;      // rows [valid, 64) must read as zero
           const bool first = pj == pg_lo;
-          const int buf = g & 1;
+          const int buf = n & 1;
 
-          mbar_wait(bar(BAR_S_FULL), g & 1, abort_flag, dev_status);
+          mbar_wait(bar(BAR_S_FULL), n & 1, abort_flag, dev_status);
           tc_fence_after();
           uint32_t sq[16];  // this warp's 16 tokens of its row
           float rowmax = -INFINITY;
@@ -399,7 +423,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __nv_bf
           l_run += psum;
 
           // ---- P buffer `buf` is free once PV of CTA page g-2 is done
-          if (g >= 2) mbar_wait(bar(BAR_PV_DONE0 + buf), ((g >> 1) - 1) & 1, abort_flag, dev_status);
+          if (n >= 2) mbar_wait(bar(BAR_PV_DONE0 + buf), ((n >> 1) - 1) & 1, abort_flag, dev_status);
           {
             unsigned char* prow = sm + kOffP + buf * kPBytes + lane * 128;
             const int c0w = 2 * warp, sw = lane & 7;
@@ -417,7 +441,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __nv_bf
           }
           // ---- rescale O^T by alpha (columns = query rows) once the previous PV has landed
           if (rescale) {
-            if (g >= 1) mbar_wait(bar(BAR_PV_DONE0 + ((g - 1) & 1)), ((g - 1) >> 1) & 1, abort_flag, dev_status);
+            if (n >= 1) mbar_wait(bar(BAR_PV_DONE0 + ((n - 1) & 1)), ((n - 1) >> 1) & 1, abort_flag, dev_status);
             tc_fence_after();
 #pragma unroll 1
             for (int t = 0; t < 4; ++t) {
@@ -445,8 +469,8 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __nv_bf
             partial_lse[static_cast<size_t>(slot) * SH + my_row] = l_tot > 0.f ? (m_used + log2f(l_tot)) * kLn2 : -INFINITY;
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
-        const int g_last = g - 1;
-        mbar_wait(bar(BAR_PV_DONE0 + (g_last & 1)), (g_last >> 1) & 1, abort_flag, dev_status);
+        const int n_last = n - 1;
+        mbar_wait(bar(BAR_PV_DONE0 + (n_last & 1)), (n_last >> 1) & 1, abort_flag, dev_status);
         tc_fence_after();
         float* dst = partial_o + (static_cast<size_t>(slot) * SH + rb * kRowBlock) * R + warp * 32 + lane;
 #pragma unroll 1
@@ -509,15 +533,23 @@ cudaError_t launch_decode_sm100(const transmla_params_t& p, int G, const __nv_bf
              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return cudaErrorInvalidValue;
+  // The absorbed queries as a 2-D tensor [B*S*H rows, 576 columns]; one box = 32 rows x 64 columns.
+  CUtensorMap qmap;
+  const int SH = p.q_len * p.num_heads;
+  const cuuint64_t qdims[2] = {static_cast<cuuint64_t>(K), static_cast<cuuint64_t>(p.batch) * SH};
+  const cuuint32_t qbox[2] = {64, kRowBlock};
+  if (encode(&qmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(q_hat), qdims, strides, qbox,
+             elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return cudaErrorInvalidValue;
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(decode_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  const int SH = p.q_len * p.num_heads;
   dim3 grid(G, (SH + kRowBlock - 1) / kRowBlock);
-  decode_sm100_kernel<<<grid, kThreads, kSmemBytes, stream>>>(map, q_hat, page_table, seqlens, cum, plan, partial_o,
+  decode_sm100_kernel<<<grid, kThreads, kSmemBytes, stream>>>(map, qmap, page_table, seqlens, cum, plan, partial_o,
                                                               partial_lse, dev_status, p.q_len, p.num_heads, p.num_pages,
                                                               p.max_pages_per_seq, p.softmax_scale * kLog2e);
   return cudaGetLastError();
