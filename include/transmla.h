@@ -69,7 +69,7 @@ typedef struct {
   float rope_theta;          /* RoPE base, 10000 in Eq. 1 */
 } transmla_params_t;
 
-/* Supported (r, dR) pairs: (512, 64), (128, 0), (64, 16).  dn: multiple of 16, dv: multiple of 8, both up to 256; D: multiple of 128.
+/* Supported (r, dR) pairs: (512, 64), (128, 0), (64, 16).  dn: multiple of 16, dv: multiple of 8, both up to 256; D: multiple of 256.
  * S*H <= 1024.  page_size == 64. */
 
 /* Byte offsets of the regions inside the workspace that carries results from

@@ -28,7 +28,7 @@ transmla_status_t check_shape(const transmla_params_t* p, bool need_hidden) {
   if (p->v_dim < 8 || p->v_dim > 256 || p->v_dim % 8) return TRANSMLA_ERR_SHAPE;
   if (p->batch < 1 || p->num_pages < 1 || p->max_pages_per_seq < 1) return TRANSMLA_ERR_SHAPE;
   if (p->num_partitions < 0 || p->num_partitions > (1 << 20)) return TRANSMLA_ERR_SHAPE;
-  if (need_hidden && (p->hidden_dim < 128 || p->hidden_dim % 128)) return TRANSMLA_ERR_SHAPE;
+  if (need_hidden && (p->hidden_dim < 256 || p->hidden_dim % 256)) return TRANSMLA_ERR_SHAPE;
   return TRANSMLA_OK;
 }
 

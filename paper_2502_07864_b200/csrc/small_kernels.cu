@@ -1,21 +1,35 @@
 // Plan, absorb, append and combine kernels of the absorbed-MLA decode step.
 //
 // These touch a few MB (weights, queries, split partials) against the hundreds of MB the split-KV
-// kernel streams.  They are small GEMMs with M = number of query rows or new tokens, so they run on
-// mma.sync tensor-core tiles with operands read straight from global memory or L2, and they are
-// fused into as few launches as the data dependencies allow: one "prologue" launch holds the append
-// blocks, the absorb blocks and the plan block.
+// kernel streams.  They are small GEMMs with M = number of query rows or new tokens, latency bound
+// rather than bandwidth bound, so they run on mma.sync tensor-core tiles, keep many independent
+// 16-byte loads in flight, and are fused into as few launches as the data dependencies allow: one
+// "prologue" launch holds the append blocks, the absorb blocks and the plan block.
+//
+// 16-byte operand loads: a lane (g, t) of an m16n8k16 tile needs k = 2t, 2t+1, 2t+8, 2t+9 of its row.
+// A dot product does not care in which order k is visited as long as both operands agree, so both
+// sides load the 8 consecutive elements 8t .. 8t+7 of a 32-wide k window with one uint4 and feed words
+// (x, y) to one MMA and (z, w) to the next.  Where one operand comes from shared memory instead, it
+// is stored there in the matching order (kperm below).
 #include "common.cuh"
 
 namespace transmla {
 
 __device__ __forceinline__ uint32_t ld_u32(const __nv_bfloat16* p) { return *reinterpret_cast<const uint32_t*>(p); }
+__device__ __forceinline__ uint4 ld_u128(const __nv_bfloat16* p) { return *reinterpret_cast<const uint4*>(p); }
+
+// Position, inside its 32-wide window, at which element p must sit in shared memory so that ldmatrix
+// hands out the fragment that pairs with a uint4 global load of the other operand.
+__device__ __forceinline__ int kperm(int p) { return ((p & 7) >> 1) * 8 + (p >> 3) * 2 + (p & 1); }
 
 // ------------------------------------------------------------------------------------------------
 // Split plan.  cum[b] = sum_{b'<b} ceil(L_b'/P); partition i owns flat pages
 // [floor(i*T/G), floor((i+1)*T/G)); plan row = (begin, end, sequence of first page, of last page).
-// One block of 256 threads; the scan runs in chunks of 256 sequences.
+// One block of 256 threads; the scan runs in chunks of 256 sequences; the prefix sums are kept in
+// shared memory (when they fit) for the binary searches.
 // ------------------------------------------------------------------------------------------------
+constexpr int kPlanSmemSeqs = 4096;
+
 __device__ __forceinline__ int seq_of_page(const int32_t* cum, int B, int x) {
   // the b in [0, B) with cum[b] <= x < cum[b+1]  ==  (first index with cum > x) - 1
   int lo = 0, hi = B + 1;
@@ -26,11 +40,14 @@ __device__ __forceinline__ int seq_of_page(const int32_t* cum, int B, int x) {
   return lo - 1;
 }
 
-__device__ void plan_block(const int32_t* __restrict__ seqlens, int B, int G, int32_t* cum, int32_t* plan) {
+__device__ void plan_block(const int32_t* __restrict__ seqlens, int B, int G, int32_t* cum, int32_t* plan,
+                           unsigned char* smem_raw) {
   __shared__ int warp_sums[8];
   __shared__ int carry;
+  int32_t* cum_s = reinterpret_cast<int32_t*>(smem_raw);  // [B+1] when B < kPlanSmemSeqs
+  const bool in_smem = B < kPlanSmemSeqs;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (tid == 0) { carry = 0; cum[0] = 0; }
+  if (tid == 0) { carry = 0; cum[0] = 0; if (in_smem) cum_s[0] = 0; }
   __syncthreads();
   for (int base = 0; base < B; base += 256) {
     const int b = base + tid;
@@ -44,66 +61,75 @@ __device__ void plan_block(const int32_t* __restrict__ seqlens, int B, int G, in
     int before = carry;
     for (int w = 0; w < warp; ++w) before += warp_sums[w];
     const int incl = v + before;
-    if (b < B) cum[b + 1] = incl;
+    if (b < B) { cum[b + 1] = incl; if (in_smem) cum_s[b + 1] = incl; }
     __syncthreads();
     if (tid == 255) carry = incl;
     __syncthreads();
   }
-  const long long T = cum[B];
+  const int32_t* cs = in_smem ? cum_s : cum;
+  const long long T = cs[B];
   for (int i = tid; i < G; i += 256) {
     const int p0 = static_cast<int>((static_cast<long long>(i) * T) / G);
     const int p1 = static_cast<int>((static_cast<long long>(i + 1) * T) / G);
     int b0 = -1, b1 = -1;
-    if (p1 > p0) { b0 = seq_of_page(cum, B, p0); b1 = seq_of_page(cum, B, p1 - 1); }
+    if (p1 > p0) { b0 = seq_of_page(cs, B, p0); b1 = seq_of_page(cs, B, p1 - 1); }
     reinterpret_cast<int4*>(plan)[i] = make_int4(p0, p1, b0, b1);
   }
 }
 
 // ------------------------------------------------------------------------------------------------
 // Absorb (Eq. 9 right, first line): q_hat[bs,h,:r] = W_UK_h^T q_nope[bs,h,:], q_hat[bs,h,r:] = q_pe[bs,h,:].
-// Block (h, rt) owns 128 latent columns of one head: it stages W_UK_h[:, tile] in shared memory once
-// and walks all query rows in 16-row tiles, so W_UK is read once in total.
+// Block (h, rt) owns 128 latent columns of one head: it stages W_UK_h[:, tile] and the head's query
+// rows (128 at a time) in shared memory and walks the rows in 16-row tiles, so W_UK is read once.
 // ------------------------------------------------------------------------------------------------
 constexpr int kAbsorbPitch = 128 + 8;
+constexpr int kAbsorbRows = 128;  // query rows staged per pass
 
 __device__ void absorb_block(const __nv_bfloat16* __restrict__ q_nope, const __nv_bfloat16* __restrict__ q_pe,
                              const __nv_bfloat16* __restrict__ w_uk, __nv_bfloat16* __restrict__ q_hat, int BS, int H,
                              int dn, int dR, int r, int h, int rt, unsigned char* smem_raw) {
+  const int apitch = dn + 8;
   __nv_bfloat16* w_s = reinterpret_cast<__nv_bfloat16*>(smem_raw);  // [dn][kAbsorbPitch]
+  __nv_bfloat16* a_s = w_s + dn * kAbsorbPitch;                      // [kAbsorbRows][dn + 8]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int g = lane >> 2, t4 = lane & 3;
+  const int g = lane >> 2, t4 = lane & 3, mi = lane >> 3;
   const int n0 = rt * 128, K = r + dR;
   for (int i = tid; i < dn * 16; i += 256) {
     const int k = i >> 4, c = i & 15;
     uint4 v = make_uint4(0, 0, 0, 0);
-    if (n0 + c * 8 < r) v = *reinterpret_cast<const uint4*>(w_uk + (static_cast<size_t>(h) * dn + k) * r + n0 + c * 8);
+    if (n0 + c * 8 < r) v = ld_u128(w_uk + (static_cast<size_t>(h) * dn + k) * r + n0 + c * 8);
     *reinterpret_cast<uint4*>(w_s + k * kAbsorbPitch + c * 8) = v;
   }
-  __syncthreads();
-  const int mi = lane >> 3;
-  for (int m0 = 0; m0 < BS; m0 += 16) {
-    float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-    const int r0 = m0 + g, r1 = m0 + g + 8;
-    const __nv_bfloat16* q0 = q_nope + (static_cast<size_t>(min(r0, BS - 1)) * H + h) * dn + t4 * 2;
-    const __nv_bfloat16* q1 = q_nope + (static_cast<size_t>(min(r1, BS - 1)) * H + h) * dn + t4 * 2;
-#pragma unroll 4
-    for (int ks = 0; ks < dn / 16; ++ks) {
-      uint32_t a[4];
-      a[0] = r0 < BS ? ld_u32(q0 + ks * 16) : 0u;
-      a[1] = r1 < BS ? ld_u32(q1 + ks * 16) : 0u;
-      a[2] = r0 < BS ? ld_u32(q0 + ks * 16 + 8) : 0u;
-      a[3] = r1 < BS ? ld_u32(q1 + ks * 16 + 8) : 0u;
-      uint32_t bf[4];
-      ldmatrix_x4_trans(bf, w_s + (ks * 16 + (mi & 1) * 8 + (lane & 7)) * kAbsorbPitch + warp * 16 + (mi >> 1) * 8);
-      mma_bf16_16816(acc[0], a, bf[0], bf[1]);
-      mma_bf16_16816(acc[1], a, bf[2], bf[3]);
+  const int chunks = dn / 8;
+  for (int p0 = 0; p0 < BS; p0 += kAbsorbRows) {
+    const int rows = min(kAbsorbRows, BS - p0);
+    const int rows16 = (rows + 15) & ~15;
+    __syncthreads();  // previous pass has consumed a_s
+    for (int i = tid; i < rows16 * chunks; i += 256) {
+      const int rr = i / chunks, c = i % chunks;
+      uint4 v = make_uint4(0, 0, 0, 0);
+      if (rr < rows) v = ld_u128(q_nope + (static_cast<size_t>(p0 + rr) * H + h) * dn + c * 8);
+      *reinterpret_cast<uint4*>(a_s + rr * apitch + c * 8) = v;
     }
+    __syncthreads();
+    for (int m0 = 0; m0 < rows16; m0 += 16) {
+      float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll 4
+      for (int ks = 0; ks < dn / 16; ++ks) {
+        uint32_t a[4], bf[4];
+        ldmatrix_x4(a, a_s + (m0 + (mi & 1) * 8 + (lane & 7)) * apitch + ks * 16 + (mi >> 1) * 8);
+        ldmatrix_x4_trans(bf, w_s + (ks * 16 + (mi & 1) * 8 + (lane & 7)) * kAbsorbPitch + warp * 16 + (mi >> 1) * 8);
+        mma_bf16_16816(acc[0], a, bf[0], bf[1]);
+        mma_bf16_16816(acc[1], a, bf[2], bf[3]);
+      }
+      const int r0 = p0 + m0 + g, r1 = r0 + 8;
 #pragma unroll
-    for (int j = 0; j < 2; ++j) {
-      const int col = n0 + warp * 16 + j * 8 + t4 * 2;
-      if (col < r) {
-        if (r0 < BS) *reinterpret_cast<uint32_t*>(q_hat + (static_cast<size_t>(r0) * H + h) * K + col) = pack_bf16(acc[j][0], acc[j][1]);
-        if (r1 < BS) *reinterpret_cast<uint32_t*>(q_hat + (static_cast<size_t>(r1) * H + h) * K + col) = pack_bf16(acc[j][2], acc[j][3]);
+      for (int j = 0; j < 2; ++j) {
+        const int col = n0 + warp * 16 + j * 8 + t4 * 2;
+        if (col < r) {
+          if (r0 < BS) *reinterpret_cast<uint32_t*>(q_hat + (static_cast<size_t>(r0) * H + h) * K + col) = pack_bf16(acc[j][0], acc[j][1]);
+          if (r1 < BS) *reinterpret_cast<uint32_t*>(q_hat + (static_cast<size_t>(r1) * H + h) * K + col) = pack_bf16(acc[j][2], acc[j][3]);
+        }
       }
     }
   }
@@ -117,64 +143,86 @@ __device__ void absorb_block(const __nv_bfloat16* __restrict__ q_nope, const __n
   }
 }
 
+static size_t absorb_smem(int dn) {
+  return (static_cast<size_t>(dn) * kAbsorbPitch + static_cast<size_t>(kAbsorbRows) * (dn + 8)) * sizeof(__nv_bfloat16);
+}
+
 // ------------------------------------------------------------------------------------------------
 // Latent append (Eq. 7 left): y = [W_DKV; W_KR] x, RoPE (Eq. 1) on y[r:], bf16, scatter to the page slot.
 // One block owns 8 consecutive output features (a RoPE pair never straddles blocks); its 8 warps
 // split the hidden dimension and meet in shared memory.  Tokens are the M dimension of the tiles.
 // Token (b, s) sits at position pos_base[b] + pos_shift + s.
 // ------------------------------------------------------------------------------------------------
-constexpr int kAppendMT = 8;  // 16-token tiles per pass
+constexpr int kAppendMaxMT = 8;  // 16-token tiles per pass
+constexpr size_t kAppendSmem = 8 * kAppendMaxMT * 16 * 8 * sizeof(float);  // 32 KB
+
+// Partial products of one warp over its slice of the hidden dimension for tokens [t0, t0 + 16*MT).
+template <int MT, int UNROLL>
+__device__ __forceinline__ void append_partial(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ wrow,
+                                               int D, int T, int t0, int k_lo, int slice, int g, int t4,
+                                               float (&acc)[kAppendMaxMT][4]) {
+  const __nv_bfloat16* xr[MT][2];
+  bool ok[MT][2];
+#pragma unroll
+  for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+    for (int hf = 0; hf < 2; ++hf) {
+      const int row = t0 + mt * 16 + g + hf * 8;
+      ok[mt][hf] = row < T;
+      xr[mt][hf] = x + static_cast<size_t>(min(row, T - 1)) * D + k_lo + t4 * 8;
+    }
+#pragma unroll UNROLL
+  for (int k = 0; k < slice; k += 32) {
+    const uint4 wv = ld_u128(wrow + k);
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+      uint4 x0 = make_uint4(0, 0, 0, 0), x1 = make_uint4(0, 0, 0, 0);
+      if (ok[mt][0]) x0 = ld_u128(xr[mt][0] + k);
+      if (ok[mt][1]) x1 = ld_u128(xr[mt][1] + k);
+      const uint32_t a0[4] = {x0.x, x1.x, x0.y, x1.y}, a1[4] = {x0.z, x1.z, x0.w, x1.w};
+      mma_bf16_16816(acc[mt], a0, wv.x, wv.y);
+      mma_bf16_16816(acc[mt], a1, wv.z, wv.w);
+    }
+  }
+}
 
 __device__ void append_block(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w,
                              const int32_t* __restrict__ pos_base, int pos_shift,
                              const int32_t* __restrict__ page_table, __nv_bfloat16* __restrict__ cache,
                              int32_t* dev_status, int B, int S, int D, int r, int dR, int num_pages, int max_pages,
                              float theta, int nb, unsigned char* smem_raw) {
-  float* red = reinterpret_cast<float*>(smem_raw);  // [8 warps][kAppendMT*16 rows][8]
+  float* red = reinterpret_cast<float*>(smem_raw);  // [8 warps][128 rows][8]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, t4 = lane & 3;
   const int K = r + dR, f0 = nb * 8, T = B * S;
   const int slice = D / 8, k_lo = warp * slice;
-  const __nv_bfloat16* wrow = w + static_cast<size_t>(f0 + g) * D + k_lo + t4 * 2;
-  for (int t0 = 0; t0 < T; t0 += kAppendMT * 16) {
-    float acc[kAppendMT][4];
+  const __nv_bfloat16* wrow = w + static_cast<size_t>(f0 + g) * D + k_lo + t4 * 8;
+  for (int t0 = 0; t0 < T; t0 += kAppendMaxMT * 16) {
+    float acc[kAppendMaxMT][4];
 #pragma unroll
-    for (int mt = 0; mt < kAppendMT; ++mt) acc[mt][0] = acc[mt][1] = acc[mt][2] = acc[mt][3] = 0.f;
-#pragma unroll 2
-    for (int k = 0; k < slice; k += 16) {
-      const uint32_t b0 = ld_u32(wrow + k), b1 = ld_u32(wrow + k + 8);
-#pragma unroll
-      for (int mt = 0; mt < kAppendMT; ++mt) {
-        if (t0 + mt * 16 < T) {
-          const int r0 = t0 + mt * 16 + g, r1 = r0 + 8;
-          const __nv_bfloat16* x0 = x + static_cast<size_t>(min(r0, T - 1)) * D + k_lo + k + t4 * 2;
-          const __nv_bfloat16* x1 = x + static_cast<size_t>(min(r1, T - 1)) * D + k_lo + k + t4 * 2;
-          uint32_t a[4];
-          a[0] = r0 < T ? ld_u32(x0) : 0u;
-          a[1] = r1 < T ? ld_u32(x1) : 0u;
-          a[2] = r0 < T ? ld_u32(x0 + 8) : 0u;
-          a[3] = r1 < T ? ld_u32(x1 + 8) : 0u;
-          mma_bf16_16816(acc[mt], a, b0, b1);
-        }
-      }
-    }
+    for (int mt = 0; mt < kAppendMaxMT; ++mt) acc[mt][0] = acc[mt][1] = acc[mt][2] = acc[mt][3] = 0.f;
+    const int left = T - t0;
+    if (left <= 16) append_partial<1, 8>(x, wrow, D, T, t0, k_lo, slice, g, t4, acc);
+    else if (left <= 32) append_partial<2, 4>(x, wrow, D, T, t0, k_lo, slice, g, t4, acc);
+    else if (left <= 64) append_partial<4, 2>(x, wrow, D, T, t0, k_lo, slice, g, t4, acc);
+    else append_partial<8, 1>(x, wrow, D, T, t0, k_lo, slice, g, t4, acc);
     __syncthreads();  // previous pass has consumed `red`
 #pragma unroll
-    for (int mt = 0; mt < kAppendMT; ++mt) {
-      if (t0 + mt * 16 < T) {
-        float* d = red + (warp * kAppendMT * 16 + mt * 16 + g) * 8 + t4 * 2;
+    for (int mt = 0; mt < kAppendMaxMT; ++mt) {
+      if (mt * 16 < left) {
+        float* d = red + (warp * kAppendMaxMT * 16 + mt * 16 + g) * 8 + t4 * 2;
         *reinterpret_cast<float2*>(d) = make_float2(acc[mt][0], acc[mt][1]);
         *reinterpret_cast<float2*>(d + 64) = make_float2(acc[mt][2], acc[mt][3]);
       }
     }
     __syncthreads();
-    const int rows = min(kAppendMT * 16, T - t0);
+    const int rows = min(kAppendMaxMT * 16, left);
     for (int i = tid; i < rows * 4; i += 256) {
       const int row = i >> 2, pr = i & 3;
       float re = 0.f, im = 0.f;
 #pragma unroll
       for (int wv = 0; wv < 8; ++wv) {
-        const float2 v = *reinterpret_cast<const float2*>(red + (wv * kAppendMT * 16 + row) * 8 + pr * 2);
+        const float2 v = *reinterpret_cast<const float2*>(red + (wv * kAppendMaxMT * 16 + row) * 8 + pr * 2);
         re += v.x; im += v.y;
       }
       const int t = t0 + row, b = t / S, s = t % S;
@@ -203,8 +251,6 @@ __device__ void append_block(const __nv_bfloat16* __restrict__ x, const __nv_bfl
   }
 }
 
-constexpr size_t kAppendSmem = 8 * kAppendMT * 16 * 8 * sizeof(float);  // 32 KB
-
 __global__ void __launch_bounds__(256) append_kernel(const __nv_bfloat16* __restrict__ x,
                                                      const __nv_bfloat16* __restrict__ w,
                                                      const int32_t* __restrict__ positions,
@@ -231,11 +277,11 @@ __global__ void __launch_bounds__(256) absorb_plan_kernel(const __nv_bfloat16* _
   if (static_cast<int>(blockIdx.x) < n_absorb) {
     absorb_block(q_nope, q_pe, w_uk, q_hat, B * S, H, dn, dR, r, blockIdx.x / r_tiles, blockIdx.x % r_tiles, smem_raw);
   } else {
-    plan_block(seqlens, B, G, cum, plan);
+    plan_block(seqlens, B, G, cum, plan, smem_raw);
   }
 }
 
-// The whole prologue of a decode step in one launch: append blocks, absorb blocks, plan block.
+// The whole prologue of a decode step in one launch: plan block, append blocks, absorb blocks.
 // The appended token of sequence b sits at seqlens[b] - S + s.
 __global__ void __launch_bounds__(256) prologue_kernel(
     const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w_dkv_kr,
@@ -246,20 +292,19 @@ __global__ void __launch_bounds__(256) prologue_kernel(
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int n_append = (r + dR) / 8;
   const int r_tiles = (r + 127) / 128;
-  const int n_absorb = H * r_tiles;
-  const int bid = blockIdx.x;
-  if (bid < n_append) {
+  const int bid = static_cast<int>(blockIdx.x) - 1;
+  if (bid < 0) {
+    plan_block(seqlens, B, G, cum, plan, smem_raw);
+  } else if (bid < n_append) {
     append_block(x, w_dkv_kr, seqlens, -S, page_table, cache, dev_status, B, S, D, r, dR, num_pages, max_pages, theta,
                  bid, smem_raw);
-  } else if (bid < n_append + n_absorb) {
+  } else {
     const int a = bid - n_append;
     absorb_block(q_nope, q_pe, w_uk, q_hat, B * S, H, dn, dR, r, a / r_tiles, a % r_tiles, smem_raw);
-  } else {
-    plan_block(seqlens, B, G, cum, plan);
   }
 }
 
-static size_t absorb_smem(int dn) { return static_cast<size_t>(dn) * kAbsorbPitch * sizeof(__nv_bfloat16); }
+constexpr int kPrologueMaxSmem = 144 * 1024;
 
 cudaError_t launch_append(const transmla_params_t& p, const __nv_bfloat16* x, const __nv_bfloat16* w,
                           const int32_t* positions, const int32_t* page_table, __nv_bfloat16* cache,
@@ -274,10 +319,11 @@ cudaError_t launch_append(const transmla_params_t& p, const __nv_bfloat16* x, co
 cudaError_t launch_absorb_plan(const transmla_params_t& p, int G, const __nv_bfloat16* q_nope,
                                const __nv_bfloat16* q_pe, const __nv_bfloat16* w_uk, __nv_bfloat16* q_hat,
                                const int32_t* seqlens, int32_t* cum, int32_t* plan, cudaStream_t stream) {
-  const size_t smem = absorb_smem(p.qk_nope_dim);
-  static bool attr_set = false;  // 68 KB at dn = 256 exceeds the default dynamic shared memory limit
+  size_t smem = absorb_smem(p.qk_nope_dim);
+  if (smem < kPlanSmemSeqs * sizeof(int32_t)) smem = kPlanSmemSeqs * sizeof(int32_t);
+  static bool attr_set = false;  // above the default dynamic shared memory limit
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(absorb_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 72 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(absorb_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPrologueMaxSmem);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
@@ -296,11 +342,11 @@ cudaError_t launch_prologue(const transmla_params_t& p, int G, const __nv_bfloat
   if (smem < kAppendSmem) smem = kAppendSmem;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(prologue_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 72 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(prologue_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPrologueMaxSmem);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  const int blocks = (p.kv_lora_rank + p.qk_rope_dim) / 8 + p.num_heads * ((p.kv_lora_rank + 127) / 128) + 1;
+  const int blocks = 1 + (p.kv_lora_rank + p.qk_rope_dim) / 8 + p.num_heads * ((p.kv_lora_rank + 127) / 128);
   prologue_kernel<<<blocks, 256, smem, stream>>>(x, w_dkv_kr, page_table, cache, q_nope, q_pe, w_uk, q_hat, seqlens, cum,
                                                  plan, dev_status, p.batch, p.q_len, p.num_heads, p.hidden_dim,
                                                  p.qk_nope_dim, p.qk_rope_dim, p.kv_lora_rank, p.num_pages,
@@ -309,11 +355,14 @@ cudaError_t launch_prologue(const transmla_params_t& p, int G, const __nv_bfloat
 }
 
 // ------------------------------------------------------------------------------------------------
-// Combine + up-projection (Eq. 9 right, last line before W_O).  Block = one head x 16 query rows.
-// Phase 1: each warp merges the split partials of two rows by their lse (segments of sequence b live
+// Combine + up-projection (Eq. 9 right, last line before W_O).  Block = one head x 8 or 16 query rows
+// x (optionally) one half of the dv output columns.
+// Phase 1: each warp merges the split partials of its rows by their lse (segments of sequence b live
 // in slots i + b for the partitions i that overlap its pages) into shared memory as a bf16 hi/lo
-// pair, so that the tensor-core product of phase 2 carries fp32-like precision of o_hat.
-// Phase 2: out[rows, h, :] = o_hat W_UV_h^T with W_UV_h read straight from global memory.
+// pair, so that the tensor-core product of phase 2 carries fp32-like precision of o_hat.  The merged
+// row is stored in kperm order.
+// Phase 2: out[rows, h, :] = o_hat W_UV_h^T with W_UV_h read straight from global memory, 16 bytes per
+// lane and all loads of a tile in flight together.
 // ------------------------------------------------------------------------------------------------
 constexpr int kCombineRows = 16;
 
@@ -362,19 +411,29 @@ __global__ void __launch_bounds__(256) combine_kernel(const int32_t* __restrict_
             const float wgt = l > -INFINITY ? __expf(l - m) : 0.f;
             den += wgt;
             const int cnt = min(32, nseg - base);
-            for (int j = 0; j < cnt; ++j) {
-              const float wj = __shfl_sync(0xffffffffu, wgt, j);
-              if (wj == 0.f) continue;
-              const float* po = partial_o + (static_cast<size_t>(i_first + base + j + b) * SH + row) * r;
+            const float* po0 = partial_o + (static_cast<size_t>(i_first + base + b) * SH + row) * r + lane * 4;
+            const size_t seg_stride = static_cast<size_t>(SH) * r;
+            // four segments per round so that their loads overlap; a zero weight skips the (unwritten) slot
+            for (int j0 = 0; j0 < cnt; j0 += 4) {
+              float wj[4];
+              float4 v[4][4];
 #pragma unroll
-              for (int c = 0; c < 4; ++c) {
-                const int k = c * 128 + lane * 4;
-                if (k < r) {
-                  const float4 v = *reinterpret_cast<const float4*>(po + k);
-                  acc[c][0] = fmaf(wj, v.x, acc[c][0]); acc[c][1] = fmaf(wj, v.y, acc[c][1]);
-                  acc[c][2] = fmaf(wj, v.z, acc[c][2]); acc[c][3] = fmaf(wj, v.w, acc[c][3]);
+              for (int u = 0; u < 4; ++u) {
+                wj[u] = (j0 + u < cnt) ? __shfl_sync(0xffffffffu, wgt, (j0 + u) & 31) : 0.f;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                  v[u][c] = make_float4(0.f, 0.f, 0.f, 0.f);
+                  if (wj[u] != 0.f && c * 128 + lane * 4 < r)
+                    v[u][c] = *reinterpret_cast<const float4*>(po0 + (j0 + u) * seg_stride + c * 128);
                 }
               }
+#pragma unroll
+              for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                  acc[c][0] = fmaf(wj[u], v[u][c].x, acc[c][0]); acc[c][1] = fmaf(wj[u], v[u][c].y, acc[c][1]);
+                  acc[c][2] = fmaf(wj[u], v[u][c].z, acc[c][2]); acc[c][3] = fmaf(wj[u], v[u][c].w, acc[c][3]);
+                }
             }
           }
 #pragma unroll
@@ -383,7 +442,7 @@ __global__ void __launch_bounds__(256) combine_kernel(const int32_t* __restrict_
           lse = m + __logf(den);
         }
       }
-      if (lse_out != nullptr && lane == 0) lse_out[(static_cast<size_t>(b) * S + s) * H + h] = lse;
+      if (lse_out != nullptr && lane == 0 && blockIdx.z == 0) lse_out[(static_cast<size_t>(b) * S + s) * H + h] = lse;
     }
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
@@ -395,26 +454,42 @@ __global__ void __launch_bounds__(256) combine_kernel(const int32_t* __restrict_
           v[e] = acc[c][e] * inv;
           lo[e] = v[e] - __bfloat162float(__float2bfloat16_rn(v[e]));
         }
-        *reinterpret_cast<uint2*>(o_hi + rr * pitch + k) = make_uint2(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]));
-        *reinterpret_cast<uint2*>(o_lo + rr * pitch + k) = make_uint2(pack_bf16(lo[0], lo[1]), pack_bf16(lo[2], lo[3]));
+        const int win = k & ~31, p = k & 31;  // elements p..p+3 of the window: two pairs, each stays adjacent
+        const int q0 = win + kperm(p), q1 = win + kperm(p + 2);
+        *reinterpret_cast<uint32_t*>(o_hi + rr * pitch + q0) = pack_bf16(v[0], v[1]);
+        *reinterpret_cast<uint32_t*>(o_hi + rr * pitch + q1) = pack_bf16(v[2], v[3]);
+        *reinterpret_cast<uint32_t*>(o_lo + rr * pitch + q0) = pack_bf16(lo[0], lo[1]);
+        *reinterpret_cast<uint32_t*>(o_lo + rr * pitch + q1) = pack_bf16(lo[2], lo[3]);
       }
     }
   }
   __syncthreads();
 
   const int g = lane >> 2, t4 = lane & 3, mi = lane >> 3;
-  for (int nt = warp; nt < dv / 8; nt += 8) {
+  const int tiles = dv / 8, tiles_per_z = (tiles + gridDim.z - 1) / gridDim.z;
+  const int nt_lo = blockIdx.z * tiles_per_z, nt_hi = min(tiles, nt_lo + tiles_per_z);
+  for (int nt = nt_lo + warp; nt < nt_hi; nt += 8) {
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
-    const __nv_bfloat16* wrow = w_uv + (static_cast<size_t>(h) * dv + nt * 8 + g) * r + t4 * 2;
-#pragma unroll 4
-    for (int ks = 0; ks < r / 16; ++ks) {
-      const uint32_t b0 = ld_u32(wrow + ks * 16), b1 = ld_u32(wrow + ks * 16 + 8);
-      uint32_t ah[4], al[4];
-      const int off = ((mi & 1) * 8 + (lane & 7)) * pitch + ks * 16 + (mi >> 1) * 8;
-      ldmatrix_x4(ah, o_hi + off);
-      ldmatrix_x4(al, o_lo + off);
-      mma_bf16_16816(acc, ah, b0, b1);
-      mma_bf16_16816(acc, al, b0, b1);
+    const __nv_bfloat16* wrow = w_uv + (static_cast<size_t>(h) * dv + nt * 8 + g) * r + t4 * 8;
+    for (int w0 = 0; w0 < r; w0 += 256) {  // up to 8 windows of 32 per round, all their loads in flight together
+      uint4 wv[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) wv[u] = (w0 + u * 32 < r) ? ld_u128(wrow + w0 + u * 32) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        if (w0 + u * 32 < r) {
+          uint32_t ah[4], al[4];
+          const int off = ((mi & 1) * 8 + (lane & 7)) * pitch + w0 + u * 32 + (mi >> 1) * 8;
+          ldmatrix_x4(ah, o_hi + off);
+          ldmatrix_x4(al, o_lo + off);
+          mma_bf16_16816(acc, ah, wv[u].x, wv[u].y);
+          mma_bf16_16816(acc, al, wv[u].x, wv[u].y);
+          ldmatrix_x4(ah, o_hi + off + 16);
+          ldmatrix_x4(al, o_lo + off + 16);
+          mma_bf16_16816(acc, ah, wv[u].z, wv[u].w);
+          mma_bf16_16816(acc, al, wv[u].z, wv[u].w);
+        }
+      }
     }
     const int col = nt * 8 + t4 * 2;
     const int bs_a = bs0 + g, bs_b = bs0 + g + 8;
@@ -430,7 +505,8 @@ cudaError_t launch_combine(const transmla_params_t& p, int G, const int32_t* cum
                            cudaStream_t stream) {
   const int BS = p.batch * p.q_len;
   const int rows = BS <= 64 ? 8 : 16;  // smaller blocks when there are few query rows, for more parallelism
-  dim3 grid(p.num_heads, (BS + rows - 1) / rows);
+  const int zsplit = (BS <= 64 && p.v_dim >= 128) ? 2 : 1;
+  dim3 grid(p.num_heads, (BS + rows - 1) / rows, zsplit);
   const size_t smem = 2 * kCombineRows * (p.kv_lora_rank + 8) * sizeof(__nv_bfloat16);
   combine_kernel<<<grid, 256, smem, stream>>>(cum, partial_o, partial_lse, w_uv, out, lse_out, p.batch, p.q_len,
                                               p.num_heads, p.kv_lora_rank, p.v_dim, G, rows);
