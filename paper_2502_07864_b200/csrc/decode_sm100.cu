@@ -321,37 +321,44 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
       const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
       const int my_row = rb * kRowBlock + lane;  // query row of this thread (same in all four replicas)
       int g = 0, n = 0;  // ring items and pages handled so far
-      for (int b = pl.z; b <= pl.w; ++b) {
+      // Q_hat rows of the next ring item: shared memory (swizzled sub-tiles of 32 rows x 128 bytes) -> this
+      // warp's replica in tensor memory, 32 columns (64 elements) at a time; then the stage is handed back.
+      auto stage_queries = [&]() {
+        const int stage = g % kStages, use = g / kStages;
+        mbar_wait(bar(BAR_KV_FULL + stage), use & 1, abort_flag, dev_status);
+        const unsigned char* qrow = sm + kOffStage + stage * kStageBytes + lane * 128;
+#pragma unroll 1
+        for (int c = 0; c < kChunks; ++c) {
+          uint32_t v[32];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const uint4 x = *reinterpret_cast<const uint4*>(qrow + c * kQTileBytes + ((j ^ (lane & 7)) << 4));
+            v[4 * j] = x.x; v[4 * j + 1] = x.y; v[4 * j + 2] = x.z; v[4 * j + 3] = x.w;
+          }
+          tmem_st32(tmem + lane_base + kColQ + c * 32, v);
+        }
+        tc_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar(BAR_Q_READY));
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (tid == 0) mbar_arrive(bar(BAR_KV_EMPTY + stage));
+        ++g;
+      };
+      auto next_segment = [&](int b) -> int {  // first sequence after b that has pages in this partition, or pl.w + 1
+        for (++b; b <= pl.w; ++b) {
+          const int c0 = cum[b];
+          if (min(pl.y, cum[b + 1]) > max(pl.x, c0)) break;
+        }
+        return b;
+      };
+      int b = next_segment(pl.z - 1);
+      if (b <= pl.w) stage_queries();
+      while (b <= pl.w) {
         const int c0 = cum[b];
         const int pg_lo = max(pl.x, c0) - c0, pg_hi = min(pl.y, cum[b + 1]) - c0;
-        if (pg_hi <= pg_lo) continue;
         const int L = seqlens[b];
         const int slot = part + b;
         const int n_vis = my_row < SH ? L - (S - 1 - my_row / H) : 0;
-
-        // ---- Q_hat rows: shared memory (swizzled sub-tiles of 32 rows x 128 bytes) -> this warp's replica in
-        //      tensor memory, 32 columns (64 elements) at a time; then the ring stage is handed back
-        {
-          const int stage = g % kStages, use = g / kStages;
-          mbar_wait(bar(BAR_KV_FULL + stage), use & 1, abort_flag, dev_status);
-          const unsigned char* qrow = sm + kOffStage + stage * kStageBytes + lane * 128;
-#pragma unroll 1
-          for (int c = 0; c < kChunks; ++c) {
-            uint32_t v[32];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              const uint4 x = *reinterpret_cast<const uint4*>(qrow + c * kQTileBytes + ((j ^ (lane & 7)) << 4));
-              v[4 * j] = x.x; v[4 * j + 1] = x.y; v[4 * j + 2] = x.z; v[4 * j + 3] = x.w;
-            }
-            tmem_st32(tmem + lane_base + kColQ + c * 32, v);
-          }
-          tc_wait_st();
-          tc_fence_before();
-          mbar_arrive(bar(BAR_Q_READY));
-          asm volatile("bar.sync 1, 128;" ::: "memory");
-          if (tid == 0) mbar_arrive(bar(BAR_KV_EMPTY + stage));
-          ++g;
-        }
 
         float m_used = -INFINITY, l_run = 0.f;
         for (int pj = pg_lo; pj < pg_hi; ++pj, ++g, ++n) {
@@ -469,6 +476,10 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
             partial_lse[static_cast<size_t>(slot) * SH + my_row] = l_tot > 0.f ? (m_used + log2f(l_tot)) * kLn2 : -INFINITY;
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
+        // The queries of the next segment go to tensor memory now (every QK^T of this segment has completed), so
+        // that its first QK^T runs while this segment's result is written out.
+        const int b_next = next_segment(b);
+        if (b_next <= pl.w) stage_queries();
         const int n_last = n - 1;
         mbar_wait(bar(BAR_PV_DONE0 + (n_last & 1)), (n_last >> 1) & 1, abort_flag, dev_status);
         tc_fence_after();
@@ -484,6 +495,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
         }
         tc_fence_before();
         asm volatile("bar.sync 1, 128;" ::: "memory");  // inv_l / l_part are reused by the next segment
+        b = b_next;
       }
     }
   }
