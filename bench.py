@@ -210,8 +210,11 @@ def run_ours(args, name, shape, seqlens, seed):
         step(i)
     barrier()
 
-    kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    for a, b_ in kev:       # create the underlying CUDA events before handing them to the library
+    # The split-KV kernel is timed by events the library records around it, on every 8th step of the timed
+    # region only: an event record between two kernels switches off their launch overlap for that step.
+    sampled = list(range(0, args.steps, 8))
+    kev = {i: (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for i in sampled}
+    for a, b_ in kev.values():       # create the underlying CUDA events before handing them to the library
         a.record(stream); b_.record(stream)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler = ClockSampler(local) if rank == 0 else None
@@ -219,13 +222,13 @@ def run_ours(args, name, shape, seqlens, seed):
     t0 = time.perf_counter()
     e0.record(stream)
     for i in range(args.steps):
-        step(i, kev[i])
+        step(i, kev.get(i))
     e1.record(stream)
     barrier()
     t1 = time.perf_counter()
     ms_total = e0.elapsed_time(e1)
     clocks = sampler.stop(t0, t1) if sampler else None
-    kernel_ms = statistics.mean(a.elapsed_time(b_) for a, b_ in kev)
+    kernel_ms = statistics.mean(a.elapsed_time(b_) for a, b_ in kev.values())
     assert int(status.item()) == 0, 'device status word set'
 
     # end to end through the host-buffer entry point: pinned host inputs, result read back every step
@@ -279,7 +282,7 @@ def run_ours(args, name, shape, seqlens, seed):
                    'parallelism': f'replicas x{world}, no data-path collective'},
         'cache_gbs': world * cache_bytes / (ms_step * 1e-3) / 1e9,
         'cache_gbs_pct_of_8tbs': 100.0 * cache_bytes / (ms_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
-        'decode_kernel_us': kernel_ms * 1e3,
+        'decode_kernel_us': kernel_ms * 1e3, 'decode_kernel_launches_timed': len(kev),
         'roofline': {'bound': 'hbm', 'achieved': achieved, 'peak': peak, 'unit': 'GB/s', 'frac': achieved / peak,
                      'peak_kind': f'{peak_kind} copy bandwidth', 'frac_of_8tbs': achieved / NOMINAL_HBM_GBS,
                      'kernel': 'split-KV decode', 'algorithmic_bytes_per_launch': algo_bytes, 'traffic': traffic},

@@ -46,6 +46,8 @@ decode_generic_kernel(const __nv_bfloat16* __restrict__ q_hat, const __nv_bfloat
   const int wk = warp & 3, wn = warp >> 2;
   const int part = blockIdx.x, rb = blockIdx.y;
   const int SH = S * H;
+  pdl_trigger();
+  pdl_wait();
   const int4 pl = reinterpret_cast<const int4*>(plan)[part];
   if (pl.y <= pl.x) return;
 
@@ -274,10 +276,9 @@ static cudaError_t launch_one(const transmla_params_t& p, int G, const __nv_bflo
   }
   const int SH = p.q_len * p.num_heads;
   dim3 grid(G, (SH + kRowBlock - 1) / kRowBlock);
-  kern<<<grid, 256, C::smem_bytes, stream>>>(q_hat, cache, page_table, seqlens, cum, plan, partial_o, partial_lse,
-                                             dev_status, p.q_len, p.num_heads, p.num_pages, p.max_pages_per_seq,
-                                             p.softmax_scale * kLog2e);
-  return cudaGetLastError();
+  return launch_pdl(kern, grid, dim3(256), C::smem_bytes, stream, q_hat, cache, page_table, seqlens, cum, plan, partial_o,
+                    partial_lse, dev_status, p.q_len, p.num_heads, p.num_pages, p.max_pages_per_seq,
+                    p.softmax_scale * kLog2e);
 }
 
 cudaError_t launch_decode_generic(const transmla_params_t& p, int G, const __nv_bfloat16* q_hat,

@@ -196,9 +196,11 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int part = blockIdx.x, rb = blockIdx.y;
   const int SH = S * H;
-  const int4 pl = reinterpret_cast<const int4*>(plan)[part];
+  pdl_trigger();
 
   if (tid == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&cache_map)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&q_map)) : "memory");
     for (int i = 0; i < kStages; ++i) { mbar_init(bar(BAR_KV_FULL + i), 1); mbar_init(bar(BAR_KV_EMPTY + i), 1); }
     mbar_init(bar(BAR_Q_READY), 128);
     mbar_init(bar(BAR_S_FULL), 1);
@@ -218,6 +220,8 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_base_s;
+  pdl_wait();  // the plan, the absorbed queries and the appended cache rows come from the kernel before this one
+  const int4 pl = reinterpret_cast<const int4*>(plan)[part];
 
   if (pl.y > pl.x) {
     if (warp == 4) {
@@ -561,10 +565,9 @@ cudaError_t launch_decode_sm100(const transmla_params_t& p, int G, const __nv_bf
     attr_set = true;
   }
   dim3 grid(G, (SH + kRowBlock - 1) / kRowBlock);
-  decode_sm100_kernel<<<grid, kThreads, kSmemBytes, stream>>>(map, qmap, page_table, seqlens, cum, plan, partial_o,
-                                                              partial_lse, dev_status, p.q_len, p.num_heads, p.num_pages,
-                                                              p.max_pages_per_seq, p.softmax_scale * kLog2e);
-  return cudaGetLastError();
+  return launch_pdl(decode_sm100_kernel, grid, dim3(kThreads), static_cast<size_t>(kSmemBytes), stream, map, qmap,
+                    page_table, seqlens, cum, plan, partial_o, partial_lse, dev_status, p.q_len, p.num_heads,
+                    p.num_pages, p.max_pages_per_seq, p.softmax_scale * kLog2e);
 }
 
 }  // namespace transmla

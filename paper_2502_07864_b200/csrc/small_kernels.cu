@@ -47,6 +47,7 @@ __device__ void plan_block(const int32_t* __restrict__ seqlens, int B, int G, in
   int32_t* cum_s = reinterpret_cast<int32_t*>(smem_raw);  // [B+1] when B < kPlanSmemSeqs
   const bool in_smem = B < kPlanSmemSeqs;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  pdl_wait();
   if (tid == 0) { carry = 0; cum[0] = 0; if (in_smem) cum_s[0] = 0; }
   __syncthreads();
   for (int base = 0; base < B; base += 256) {
@@ -100,11 +101,12 @@ __device__ void absorb_block(const __nv_bfloat16* __restrict__ q_nope, const __n
     if (n0 + c * 8 < r) v = ld_u128(w_uk + (static_cast<size_t>(h) * dn + k) * r + n0 + c * 8);
     *reinterpret_cast<uint4*>(w_s + k * kAbsorbPitch + c * 8) = v;
   }
+  pdl_wait();  // the queries may come from the kernel before this one; the weights above may not
   const int chunks = dn / 8;
   for (int p0 = 0; p0 < BS; p0 += kAbsorbRows) {
     const int rows = min(kAbsorbRows, BS - p0);
     const int rows16 = (rows + 15) & ~15;
-    __syncthreads();  // previous pass has consumed a_s
+    if (p0 > 0) __syncthreads();  // previous pass has consumed a_s
     for (int i = tid; i < rows16 * chunks; i += 256) {
       const int rr = i / chunks, c = i % chunks;
       uint4 v = make_uint4(0, 0, 0, 0);
@@ -197,6 +199,9 @@ __device__ void append_block(const __nv_bfloat16* __restrict__ x, const __nv_bfl
   const int K = r + dR, f0 = nb * 8, T = B * S;
   const int slice = D / 8, k_lo = warp * slice;
   const __nv_bfloat16* wrow = w + static_cast<size_t>(f0 + g) * D + k_lo + t4 * 8;
+  if (t4 == 0)
+    for (int k = 0; k < slice; k += 64) prefetch_l2(wrow + k);  // 128-byte lines of this warp's 8 weight rows
+  pdl_wait();  // activations, positions and the cache may belong to kernels still in flight; the weights may not
   for (int t0 = 0; t0 < T; t0 += kAppendMaxMT * 16) {
     float acc[kAppendMaxMT][4];
 #pragma unroll
@@ -259,6 +264,7 @@ __global__ void __launch_bounds__(256) append_kernel(const __nv_bfloat16* __rest
                                                      int S, int D, int r, int dR, int num_pages, int max_pages,
                                                      float theta) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
+  pdl_trigger();
   append_block(x, w, positions, 0, page_table, cache, dev_status, B, S, D, r, dR, num_pages, max_pages, theta,
                blockIdx.x, smem_raw);
 }
@@ -272,6 +278,7 @@ __global__ void __launch_bounds__(256) absorb_plan_kernel(const __nv_bfloat16* _
                                                           int32_t* plan, int B, int S, int H, int dn, int dR, int r,
                                                           int G) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
+  pdl_trigger();
   const int r_tiles = (r + 127) / 128;
   const int n_absorb = H * r_tiles;
   if (static_cast<int>(blockIdx.x) < n_absorb) {
@@ -290,6 +297,7 @@ __global__ void __launch_bounds__(256) prologue_kernel(
     const int32_t* __restrict__ seqlens, int32_t* cum, int32_t* plan, int32_t* dev_status, int B, int S, int H, int D,
     int dn, int dR, int r, int num_pages, int max_pages, float theta, int G) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
+  pdl_trigger();
   const int n_append = (r + dR) / 8;
   const int r_tiles = (r + 127) / 128;
   const int bid = static_cast<int>(blockIdx.x) - 1;
@@ -310,10 +318,9 @@ cudaError_t launch_append(const transmla_params_t& p, const __nv_bfloat16* x, co
                           const int32_t* positions, const int32_t* page_table, __nv_bfloat16* cache,
                           int32_t* dev_status, cudaStream_t stream) {
   const int K = p.kv_lora_rank + p.qk_rope_dim;
-  append_kernel<<<K / 8, 256, kAppendSmem, stream>>>(x, w, positions, page_table, cache, dev_status, p.batch, p.q_len,
-                                                     p.hidden_dim, p.kv_lora_rank, p.qk_rope_dim, p.num_pages,
-                                                     p.max_pages_per_seq, p.rope_theta);
-  return cudaGetLastError();
+  return launch_pdl(append_kernel, dim3(K / 8), dim3(256), kAppendSmem, stream, x, w, positions, page_table, cache,
+                    dev_status, p.batch, p.q_len, p.hidden_dim, p.kv_lora_rank, p.qk_rope_dim, p.num_pages,
+                    p.max_pages_per_seq, p.rope_theta);
 }
 
 cudaError_t launch_absorb_plan(const transmla_params_t& p, int G, const __nv_bfloat16* q_nope,
@@ -328,9 +335,8 @@ cudaError_t launch_absorb_plan(const transmla_params_t& p, int G, const __nv_bfl
     attr_set = true;
   }
   const int blocks = p.num_heads * ((p.kv_lora_rank + 127) / 128) + 1;
-  absorb_plan_kernel<<<blocks, 256, smem, stream>>>(q_nope, q_pe, w_uk, q_hat, seqlens, cum, plan, p.batch, p.q_len,
-                                                    p.num_heads, p.qk_nope_dim, p.qk_rope_dim, p.kv_lora_rank, G);
-  return cudaGetLastError();
+  return launch_pdl(absorb_plan_kernel, dim3(blocks), dim3(256), smem, stream, q_nope, q_pe, w_uk, q_hat, seqlens, cum,
+                    plan, p.batch, p.q_len, p.num_heads, p.qk_nope_dim, p.qk_rope_dim, p.kv_lora_rank, G);
 }
 
 cudaError_t launch_prologue(const transmla_params_t& p, int G, const __nv_bfloat16* x, const __nv_bfloat16* w_dkv_kr,
@@ -347,11 +353,9 @@ cudaError_t launch_prologue(const transmla_params_t& p, int G, const __nv_bfloat
     attr_set = true;
   }
   const int blocks = 1 + (p.kv_lora_rank + p.qk_rope_dim) / 8 + p.num_heads * ((p.kv_lora_rank + 127) / 128);
-  prologue_kernel<<<blocks, 256, smem, stream>>>(x, w_dkv_kr, page_table, cache, q_nope, q_pe, w_uk, q_hat, seqlens, cum,
-                                                 plan, dev_status, p.batch, p.q_len, p.num_heads, p.hidden_dim,
-                                                 p.qk_nope_dim, p.qk_rope_dim, p.kv_lora_rank, p.num_pages,
-                                                 p.max_pages_per_seq, p.rope_theta, G);
-  return cudaGetLastError();
+  return launch_pdl(prologue_kernel, dim3(blocks), dim3(256), smem, stream, x, w_dkv_kr, page_table, cache, q_nope, q_pe,
+                    w_uk, q_hat, seqlens, cum, plan, dev_status, p.batch, p.q_len, p.num_heads, p.hidden_dim,
+                    p.qk_nope_dim, p.qk_rope_dim, p.kv_lora_rank, p.num_pages, p.max_pages_per_seq, p.rope_theta, G);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -376,9 +380,24 @@ __global__ void __launch_bounds__(256) combine_kernel(const int32_t* __restrict_
   const int pitch = r + 8;
   __nv_bfloat16* o_hi = reinterpret_cast<__nv_bfloat16*>(smem_raw);  // [16][pitch]
   __nv_bfloat16* o_lo = o_hi + kCombineRows * pitch;                 // [16][pitch]
+  pdl_trigger();
   const int h = blockIdx.x, bs0 = blockIdx.y * rows_per_block;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int SH = S * H, BS = B * S;
+  const int g = lane >> 2, t4 = lane & 3, mi = lane >> 3;
+  const int tiles = dv / 8, tiles_per_z = (tiles + gridDim.z - 1) / gridDim.z;
+  const int nt_lo = blockIdx.z * tiles_per_z, nt_hi = min(tiles, nt_lo + tiles_per_z);
+  // The weights do not depend on the merge: the first tile's 16-byte loads are issued now and land while
+  // the partials are merged.
+  constexpr int kWin = 16;  // windows of 32 columns held in registers (r <= 512 fits one round)
+  uint4 wv[kWin];
+  {
+    const int nt = nt_lo + warp;
+    const __nv_bfloat16* wrow = w_uv + (static_cast<size_t>(h) * dv + min(nt, tiles - 1) * 8 + g) * r + t4 * 8;
+#pragma unroll
+    for (int u = 0; u < kWin; ++u) wv[u] = (nt < nt_hi && u * 32 < r) ? ld_u128(wrow + u * 32) : make_uint4(0, 0, 0, 0);
+  }
+  pdl_wait();  // the partials and the prefix sums come from the kernels before this one
   const long long T = cum[B];
 
   for (int rr = warp; rr < kCombineRows; rr += 8) {
@@ -465,18 +484,17 @@ __global__ void __launch_bounds__(256) combine_kernel(const int32_t* __restrict_
   }
   __syncthreads();
 
-  const int g = lane >> 2, t4 = lane & 3, mi = lane >> 3;
-  const int tiles = dv / 8, tiles_per_z = (tiles + gridDim.z - 1) / gridDim.z;
-  const int nt_lo = blockIdx.z * tiles_per_z, nt_hi = min(tiles, nt_lo + tiles_per_z);
   for (int nt = nt_lo + warp; nt < nt_hi; nt += 8) {
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
     const __nv_bfloat16* wrow = w_uv + (static_cast<size_t>(h) * dv + nt * 8 + g) * r + t4 * 8;
-    for (int w0 = 0; w0 < r; w0 += 256) {  // up to 8 windows of 32 per round, all their loads in flight together
-      uint4 wv[8];
+    for (int w0 = 0; w0 < r; w0 += kWin * 32) {  // kWin windows per round, all their loads in flight together
+      if (nt != nt_lo + warp || w0 != 0) {
 #pragma unroll
-      for (int u = 0; u < 8; ++u) wv[u] = (w0 + u * 32 < r) ? ld_u128(wrow + w0 + u * 32) : make_uint4(0, 0, 0, 0);
+        for (int u = 0; u < kWin; ++u)
+          wv[u] = (w0 + u * 32 < r) ? ld_u128(wrow + w0 + u * 32) : make_uint4(0, 0, 0, 0);
+      }
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
+      for (int u = 0; u < kWin; ++u) {
         if (w0 + u * 32 < r) {
           uint32_t ah[4], al[4];
           const int off = ((mi & 1) * 8 + (lane & 7)) * pitch + w0 + u * 32 + (mi >> 1) * 8;
@@ -508,9 +526,8 @@ cudaError_t launch_combine(const transmla_params_t& p, int G, const int32_t* cum
   const int zsplit = (BS <= 64 && p.v_dim >= 128) ? 2 : 1;
   dim3 grid(p.num_heads, (BS + rows - 1) / rows, zsplit);
   const size_t smem = 2 * kCombineRows * (p.kv_lora_rank + 8) * sizeof(__nv_bfloat16);
-  combine_kernel<<<grid, 256, smem, stream>>>(cum, partial_o, partial_lse, w_uv, out, lse_out, p.batch, p.q_len,
-                                              p.num_heads, p.kv_lora_rank, p.v_dim, G, rows);
-  return cudaGetLastError();
+  return launch_pdl(combine_kernel, grid, dim3(256), smem, stream, cum, partial_o, partial_lse, w_uv, out, lse_out,
+                    p.batch, p.q_len, p.num_heads, p.kv_lora_rank, p.v_dim, G, rows);
 }
 
 }  // namespace transmla
