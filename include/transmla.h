@@ -48,6 +48,9 @@ typedef enum {
   TRANSMLA_ERR_ARCH = 7       /* the current device is not compute capability 10.x */
 } transmla_status_t;
 
+/* page-equivalents charged to a partition for every sequence it opens (split plan) */
+#define TRANSMLA_SEGMENT_COST_PAGES 2
+
 /* bits of the device status word */
 #define TRANSMLA_DEV_BAD_PAGE 1
 #define TRANSMLA_DEV_TIMEOUT 2
@@ -75,11 +78,13 @@ typedef struct {
 /* Byte offsets of the regions inside the workspace that carries results from
  * transmla_mla_decode to transmla_mla_combine.  All regions are written by transmla_mla_decode.
  *   q_hat       bf16  [B, S, H, r+dR]   absorbed queries (Eq. 9 right, first line)
- *   cum_pages   int32 [B+1]             cum[b] = sum_{b'<b} ceil(L_b'/P)
- *   plan        int32 [G, 4]            per partition: flat page begin, end, sequence of first page,
- *                                       sequence of last page (-1, -1 for an empty partition);
- *                                       partition i owns flat pages [floor(i*T/G), floor((i+1)*T/G)),
- *                                       T = cum[B]
+ *   cum_pages   int32 [B+1]             slot prefix sums: a sequence with n_b = ceil(L_b/P) > 0 pages owns
+ *                                       TRANSMLA_SEGMENT_COST_PAGES virtual slots followed by its n_b page
+ *                                       slots; cum[b] = number of slots before sequence b
+ *   plan        int32 [G, 4]            per partition: slot begin, end, sequence of first slot, sequence of
+ *                                       last slot (-1, -1 for an empty partition); partition i owns slots
+ *                                       [floor(i*T/G), floor((i+1)*T/G)), T = cum[B].  The virtual slots make
+ *                                       a partition that opens a second sequence shorter by that many pages
  *   partial_o   fp32  [G+B-1, S*H, r]   per segment (partition i, sequence b), slot = i + b:
  *                                       softmax-weighted mean of c_j over the segment's visible tokens
  *   partial_lse fp32  [G+B-1, S*H]      natural-log softmax denominator of the segment (-inf = empty)

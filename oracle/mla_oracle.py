@@ -152,23 +152,30 @@ def absorb(q_nope, q_pe, w_uk):
     return np.concatenate([q_lat, np.asarray(q_pe, np.float64)], axis=-1)
 
 
-def split_plan(seqlens, page_size, G):
-    """Balanced split of all cache pages of a batch over G partitions (index path).
+SEGMENT_COST_PAGES = 2   # what opening one more sequence costs a partition, in page-equivalents
 
-    Sequence b owns n_b = ceil(L_b / P) pages; pages are numbered in sequence order,
-    cum[b] = n_0 + ... + n_{b-1}, T = cum[B].  Partition i owns flat pages
-    [floor(i*T/G), floor((i+1)*T/G)).  Returned: cum [B+1] and plan [G,4] with rows
-    (flat_begin, flat_end, seq of first page, seq of last page); an empty partition has
-    seq fields -1.  Written as a plain walk over every page.
+
+def split_plan(seqlens, page_size, G, seg_cost=SEGMENT_COST_PAGES):
+    """Balanced split of all cache pages of a batch over G partitions (index path; the library's own rule).
+
+    Sequence b owns n_b = ceil(L_b / P) pages.  Every non-empty sequence is given seg_cost extra
+    "virtual" slots in front of its pages, so that a partition which has to open a second sequence
+    (load its queries, write out another partial result) receives that many fewer pages.  Slots are
+    numbered in sequence order: cum[b] = sum over b' < b of (n_b' + seg_cost if n_b' > 0 else 0),
+    T = cum[B]; page j of sequence b is slot cum[b] + seg_cost + j.  Partition i owns slots
+    [floor(i*T/G), floor((i+1)*T/G)).  Returned: cum [B+1] and plan [G,4] with rows (slot_begin,
+    slot_end, sequence of the first slot, sequence of the last slot); an empty partition has sequence
+    fields -1.  Written as a plain walk over every slot.
     """
     B = len(seqlens)
     cum = np.zeros(B + 1, dtype=np.int64)
-    for b in range(B):
-        cum[b + 1] = cum[b] + (int(seqlens[b]) + page_size - 1) // page_size
-    T = int(cum[B])
     owner_seq = []
     for b in range(B):
-        owner_seq += [b] * int(cum[b + 1] - cum[b])
+        n = (int(seqlens[b]) + page_size - 1) // page_size
+        v = n + seg_cost if n > 0 else 0
+        cum[b + 1] = cum[b] + v
+        owner_seq += [b] * v
+    T = int(cum[B])
     plan = np.zeros((G, 4), dtype=np.int32)
     for i in range(G):
         p0, p1 = (i * T) // G, ((i + 1) * T) // G
@@ -176,11 +183,11 @@ def split_plan(seqlens, page_size, G):
     return cum.astype(np.int32), plan
 
 
-def plan_segments(cum, plan):
+def plan_segments(cum, plan, seg_cost=SEGMENT_COST_PAGES):
     """Segments = maximal page ranges inside one partition and one sequence.
 
     Returns a list of (partition i, sequence b, first page in b, end page in b, slot) with
-    slot = i + b, which is distinct for distinct segments because walking the pages in order
+    slot = i + b, which is distinct for distinct segments because walking the slots in order
     moves to a new segment only by increasing i, b or both.
     """
     segs = []
@@ -189,9 +196,10 @@ def plan_segments(cum, plan):
         if p1 <= p0:
             continue
         for b in range(b0, b1 + 1):
-            lo, hi = max(p0, int(cum[b])), min(p1, int(cum[b + 1]))
+            first = int(cum[b]) + seg_cost                     # slot of page 0 of sequence b
+            lo, hi = max(p0, first), min(p1, int(cum[b + 1]))
             if hi > lo:
-                segs.append((i, b, lo - int(cum[b]), hi - int(cum[b]), i + b))
+                segs.append((i, b, lo - first, hi - first, i + b))
     return segs
 
 

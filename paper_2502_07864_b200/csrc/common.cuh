@@ -10,6 +10,7 @@ namespace transmla {
 
 constexpr int kPage = 64;       // tokens per cache page (P)
 constexpr int kRowBlock = 32;   // query rows (s*H + h) one CTA works on
+constexpr int kSegCost = TRANSMLA_SEGMENT_COST_PAGES;  // virtual slots in front of every non-empty sequence
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 

@@ -54,7 +54,7 @@ decode_generic_kernel(const __nv_bfloat16* __restrict__ q_hat, const __nv_bfloat
   const int srow = tid >> 3, ssub = tid & 7;  // softmax: 8 threads per query row, 8 tokens each
 
   for (int b = pl.z; b <= pl.w; ++b) {
-    const int c0 = cum[b];
+    const int c0 = cum[b] + kSegCost;  // slot of page 0 of sequence b
     const int pg_lo = max(pl.x, c0) - c0, pg_hi = min(pl.y, cum[b + 1]) - c0;
     if (pg_hi <= pg_lo) continue;
     const int L = seqlens[b];

@@ -28,6 +28,17 @@
 namespace transmla {
 namespace sm100 {
 
+// Optional timeline instrumentation (compile with -DTRANSMLA_TRACE): clock64 stamps of one CTA's pipeline
+// events and the global-timer start/end of every CTA, read back with transmla_trace_dump().
+#ifdef TRANSMLA_TRACE
+__device__ long long g_trace[16][256];
+#define TR(ev, idx) do { if (blockIdx.x == 3 && blockIdx.y == 0 && (idx) < 256) g_trace[ev][idx] = clock64(); } while (0)
+#define TR_GLOBAL(ev) do { long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); if (blockIdx.x < 256 && blockIdx.y == 0) g_trace[ev][blockIdx.x] = t_; } while (0)
+#else
+#define TR(ev, idx) do { } while (0)
+#define TR_GLOBAL(ev) do { } while (0)
+#endif
+
 constexpr int R = 512, DR = 64, K = R + DR;
 constexpr int kChunks = K / 64;                       // 9 sub-tiles of 64 columns (128 bytes) per page
 constexpr int kSubTileBytes = kPage * 128;            // 8192
@@ -220,6 +231,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_base_s;
+  if (tid == 0) { TR(13, 0); TR_GLOBAL(15); }
   pdl_wait();  // the plan, the absorbed queries and the appended cache rows come from the kernel before this one
   const int4 pl = reinterpret_cast<const int4*>(plan)[part];
 
@@ -231,10 +243,11 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
       auto acquire = [&](int gi) -> uint32_t {  // waits for the stage of ring item gi; returns its index
         const int stage = gi % kStages, use = gi / kStages;
         mbar_wait(bar(BAR_KV_EMPTY + stage), (use & 1) ^ 1, abort_flag, dev_status);
+        TR(0, gi);
         return stage;
       };
       for (int b = pl.z; b <= pl.w; ++b) {
-        const int c0 = cum[b];
+        const int c0 = cum[b] + kSegCost;  // slot of page 0 of sequence b
         const int pg_lo = max(pl.x, c0) - c0, pg_hi = min(pl.y, cum[b + 1]) - c0;
         if (pg_hi <= pg_lo) continue;
         {
@@ -272,6 +285,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
         auto issue_pv = [&](int gr, int gp, bool first_of_segment) {  // O^T += C^T P^T for page gp held in ring item gr
           const int stage = gr % kStages;
           mbar_wait(bar(BAR_P_READY), gp & 1, abort_flag, dev_status);
+          TR(4, gr);
           tc_fence_after();
           const uint64_t a0 = smem_desc(base + kOffStage + stage * kStageBytes, kSubTileBytes, 1024);
           const uint64_t b0 = smem_desc(base + kOffP + (gp & 1) * kPBytes, 16, 1024);
@@ -290,9 +304,10 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
             tc_commit(bar(BAR_PV_DONE0 + (gp & 1)));
           }
           __syncwarp();
+          TR(5, gr);
         };
         for (int b = pl.z; b <= pl.w; ++b) {
-          const int c0 = cum[b];
+          const int c0 = cum[b] + kSegCost;  // slot of page 0 of sequence b
           const int pg_lo = max(pl.x, c0) - c0, pg_hi = min(pl.y, cum[b + 1]) - c0;
           if (pg_hi <= pg_lo) continue;
           ++g;  // the segment's query item is consumed by the softmax warps
@@ -301,7 +316,9 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
           for (int pj = pg_lo; pj < pg_hi; ++pj, ++g, ++n) {
             const int stage = g % kStages, use = g / kStages;
             mbar_wait(bar(BAR_KV_FULL + stage), use & 1, abort_flag, dev_status);
+            TR(1, g);
             if (n > 0) mbar_wait(bar(BAR_S_FREE), (n - 1) & 1, abort_flag, dev_status);
+            TR(2, g);
             tc_fence_after();
             const uint64_t k0 = smem_desc(base + kOffStage + stage * kStageBytes, 16, 1024);
 #pragma unroll
@@ -315,6 +332,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
             }
             if (elect_one()) tc_commit(bar(BAR_S_FULL));
             __syncwarp();
+            TR(3, g);
             if (pj > pg_lo) issue_pv(g - 1, n - 1, pj - 1 == pg_lo);
           }
           issue_pv(g - 1, n - 1, pg_hi - 1 == pg_lo);
@@ -345,12 +363,12 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
         tc_fence_before();
         mbar_arrive(bar(BAR_Q_READY));
         asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (tid == 0) mbar_arrive(bar(BAR_KV_EMPTY + stage));
+        if (tid == 0) { mbar_arrive(bar(BAR_KV_EMPTY + stage)); TR(11, g); }
         ++g;
       };
       auto next_segment = [&](int b) -> int {  // first sequence after b that has pages in this partition, or pl.w + 1
         for (++b; b <= pl.w; ++b) {
-          const int c0 = cum[b];
+          const int c0 = cum[b] + kSegCost;  // slot of page 0 of sequence b
           if (min(pl.y, cum[b + 1]) > max(pl.x, c0)) break;
         }
         return b;
@@ -358,7 +376,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
       int b = next_segment(pl.z - 1);
       if (b <= pl.w) stage_queries();
       while (b <= pl.w) {
-        const int c0 = cum[b];
+        const int c0 = cum[b] + kSegCost;  // slot of page 0 of sequence b
         const int pg_lo = max(pl.x, c0) - c0, pg_hi = min(pl.y, cum[b + 1]) - c0;
         const int L = seqlens[b];
         const int slot = part + b;
@@ -374,7 +392,9 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
           const bool first = pj == pg_lo;
           const int buf = n & 1;
 
+          if (tid == 0) TR(6, g);
           mbar_wait(bar(BAR_S_FULL), n & 1, abort_flag, dev_status);
+          if (tid == 0) TR(7, g);
           tc_fence_after();
           uint32_t sq[16];  // this warp's 16 tokens of its row
           float rowmax = -INFINITY;
@@ -394,6 +414,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
           }
           tc_fence_before();
           mbar_arrive(bar(BAR_S_FREE));
+          if (tid == 0) TR(8, g);
 
           if (warp == 0) {
             // Lazy rescale: the reference maximum only moves when some row's new maximum exceeds it by 2^8.
@@ -468,6 +489,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
           fence_proxy_async();
           tc_fence_before();
           mbar_arrive(bar(BAR_P_READY));
+          if (tid == 0) TR(9, g);
         }
 
         // ---- epilogue of the segment: wait for the last PV, normalise, store O (transposed back) and lse
@@ -484,6 +506,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
         // that its first QK^T runs while this segment's result is written out.
         const int b_next = next_segment(b);
         if (b_next <= pl.w) stage_queries();
+        if (tid == 0) TR(12, g);
         const int n_last = n - 1;
         mbar_wait(bar(BAR_PV_DONE0 + (n_last & 1)), (n_last >> 1) & 1, abort_flag, dev_status);
         tc_fence_after();
@@ -499,11 +522,13 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
         }
         tc_fence_before();
         asm volatile("bar.sync 1, 128;" ::: "memory");  // inv_l / l_part are reused by the next segment
+        if (tid == 0) TR(14, g);
         b = b_next;
       }
     }
   }
 
+  if (tid == 0) { TR(13, 1); TR_GLOBAL(10); }
   // ---- teardown: everyone arrives, tensor memory is returned
   tc_fence_before();
   __syncthreads();
@@ -528,6 +553,12 @@ static PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
 }
 
 }  // namespace sm100
+
+#ifdef TRANSMLA_TRACE
+extern "C" int transmla_trace_dump(long long* host) {
+  return static_cast<int>(cudaMemcpyFromSymbol(host, sm100::g_trace, sizeof(long long) * 16 * 256));
+}
+#endif
 
 bool decode_sm100_supported(const transmla_params_t& p) { return p.kv_lora_rank == sm100::R && p.qk_rope_dim == sm100::DR; }
 

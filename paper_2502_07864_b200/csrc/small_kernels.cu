@@ -23,8 +23,9 @@ __device__ __forceinline__ uint4 ld_u128(const __nv_bfloat16* p) { return *reint
 __device__ __forceinline__ int kperm(int p) { return ((p & 7) >> 1) * 8 + (p >> 3) * 2 + (p & 1); }
 
 // ------------------------------------------------------------------------------------------------
-// Split plan.  cum[b] = sum_{b'<b} ceil(L_b'/P); partition i owns flat pages
-// [floor(i*T/G), floor((i+1)*T/G)); plan row = (begin, end, sequence of first page, of last page).
+// Split plan.  Every non-empty sequence owns ceil(L_b/P) page slots preceded by kSegCost virtual slots (the
+// price of opening a sequence); cum[b] = slots before sequence b; partition i owns slots
+// [floor(i*T/G), floor((i+1)*T/G)); plan row = (begin, end, sequence of first slot, of last slot).
 // One block of 256 threads; the scan runs in chunks of 256 sequences; the prefix sums are kept in
 // shared memory (when they fit) for the binary searches.
 // ------------------------------------------------------------------------------------------------
@@ -53,7 +54,7 @@ __device__ void plan_block(const int32_t* __restrict__ seqlens, int B, int G, in
   for (int base = 0; base < B; base += 256) {
     const int b = base + tid;
     int n = 0;
-    if (b < B) { int L = seqlens[b]; n = L > 0 ? (L + kPage - 1) / kPage : 0; }
+    if (b < B) { int L = seqlens[b]; n = L > 0 ? (L + kPage - 1) / kPage + kSegCost : 0; }
     int v = n;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) { int t = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += t; }
@@ -408,7 +409,7 @@ __global__ void __launch_bounds__(256) combine_kernel(const int32_t* __restrict_
     float lse = -INFINITY, inv = 0.f;
     if (rr < rows_per_block && bs < BS) {
       const int b = bs / S, s = bs % S, row = s * H + h;
-      const int c0 = cum[b], c1 = cum[b + 1];
+      const int c0 = cum[b] + kSegCost, c1 = cum[b + 1];  // slots of this sequence's pages
       if (c1 > c0) {
         const int i_first = static_cast<int>(((static_cast<long long>(c0) + 1) * G - 1) / T);
         const int i_last = static_cast<int>((static_cast<long long>(c1) * G - 1) / T);

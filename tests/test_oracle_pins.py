@@ -309,11 +309,12 @@ def test_empty_sequence_gives_zero_and_minus_inf():
 @pytest.mark.parametrize('seqlens,G', [((17, 64), 1), ((17, 64), 5), ((8192,) * 16, 148), ((0, 5, 0, 700, 64, 65), 7),
                                        ((1,), 4), ((0, 0), 3), ((1000, 3, 3, 3, 9000), 33)])
 def test_split_plan_properties_and_closed_form(seqlens, G):
-    P = 64
+    P, c = 64, orc.SEGMENT_COST_PAGES
     cum, plan = orc.split_plan(seqlens, P, G)
     n = [(L + P - 1) // P for L in seqlens]
-    assert list(cum) == [sum(n[:b]) for b in range(len(n) + 1)]
-    T = sum(n)
+    v = [x + c if x > 0 else 0 for x in n]
+    assert list(cum) == [sum(v[:b]) for b in range(len(n) + 1)]
+    T = sum(v)
     # partitions tile [0, T) in order with sizes differing by at most one
     assert plan[0, 0] == 0 and plan[-1, 1] == T and all(plan[i, 1] == plan[i + 1, 0] for i in range(G - 1))
     sizes = plan[:, 1] - plan[:, 0]
@@ -334,6 +335,11 @@ def test_split_plan_properties_and_closed_form(seqlens, G):
         assert slot == i + b and 0 <= slot <= G + len(n) - 2
     assert all(seen[b] == list(range(n[b])) for b in seen)
     assert len({s[4] for s in segs}) == len(segs)
+    # load per partition = pages + c per sequence opened after the first, never above the even share + c
+    load = {}
+    for (i, b, lo, hi, slot) in segs:
+        load[i] = load.get(i, -c) + (hi - lo) + c
+    assert all(x <= -(-T // G) + c for x in load.values())
 
 
 # ---------------------------------------------------------------- append (Eq. 7 left)
