@@ -167,7 +167,7 @@ def run_reference(args, name, shape, seqlens, seed):
 def run_ours(args, name, shape, seqlens, seed):
     import torch
     import torch.distributed as dist
-    from paper_2502_07864_b200 import binding, build, synth
+    from paper_2502_07864_b200 import binding, build, replicas, synth
 
     rank = int(os.environ.get('RANK', '0'))
     world = int(os.environ.get('WORLD_SIZE', '1'))
@@ -184,8 +184,8 @@ def run_ours(args, name, shape, seqlens, seed):
     B, S, H = len(seqlens), shape.S, shape.H
     scale = (shape.dn + shape.dR) ** -0.5
     n_copies = args.cache_copies
-    dc = synth.make_decode_case(shape, seqlens, seed + 100 * rank, device='cuda')
-    ac = synth.make_append_case(shape, [L - S for L in seqlens], seed + 100 * rank + 1, device='cuda')
+    dc = synth.make_decode_case(shape, seqlens, replicas.rank_seed(seed, rank), device='cuda')
+    ac = synth.make_append_case(shape, [L - S for L in seqlens], replicas.rank_seed(seed, rank) + 1, device='cuda')
     caches = [dc['cache']] + [dc['cache'].clone() for _ in range(n_copies - 1)]
     params = binding.make_params(shape, B, dc['cache'].shape[0], dc['page_table'].shape[1], scale)
     ws, lay = binding.alloc_workspace(params)
@@ -202,9 +202,7 @@ def run_ours(args, name, shape, seqlens, seed):
                                      status, stream)
 
     def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+        replicas.barrier('cuda')
 
     for i in range(max(args.warmup, 3)):
         step(i)
@@ -254,10 +252,7 @@ def run_ours(args, name, shape, seqlens, seed):
     h2d = sum(v.numel() * v.element_size() for v in h.values())
     d2h = h_out.numel() * 2 + h_lse.numel() * 4 + 4
 
-    times = torch.tensor([ms_total, e2e_s * 1e3], dtype=torch.float64, device='cuda')
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms_total, e2e_ms = (float(v) for v in times.tolist())
+    ms_total, e2e_ms = replicas.max_over_ranks([ms_total, e2e_s * 1e3], device='cuda')
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -272,7 +267,7 @@ def run_ours(args, name, shape, seqlens, seed):
     peak, peak_kind = measured_hbm_peak()
     traffic = None
     line = {
-        'metric': METRIC, 'value': tokens_per_step / (ms_step * 1e-3), 'unit': 'tokens/s', 'n_gpus': world,
+        'metric': METRIC, 'value': replicas.whole_job_rate(B * S, args.steps, ms_total), 'unit': 'tokens/s', 'n_gpus': world,
         'steps': args.steps, 'warmup': max(args.warmup, 3), 'ms_per_step': ms_step, 'higher_is_better': True,
         'scaling': 'weak', 'vs_baseline': None, 'dtype': 'bf16', 'data': 'synthetic',
         'config': {'workload': name, 'batch_per_gpu': B, 'q_len': S, 'heads': H, 'latent': shape.r, 'rope': shape.dR,
@@ -286,7 +281,7 @@ def run_ours(args, name, shape, seqlens, seed):
         'roofline': {'bound': 'hbm', 'achieved': achieved, 'peak': peak, 'unit': 'GB/s', 'frac': achieved / peak,
                      'peak_kind': f'{peak_kind} copy bandwidth', 'frac_of_8tbs': achieved / NOMINAL_HBM_GBS,
                      'kernel': 'split-KV decode', 'algorithmic_bytes_per_launch': algo_bytes, 'traffic': traffic},
-        'e2e': {'value': tokens_per_step / (e2e_ms * 1e-3 / args.steps), 'unit': 'tokens/s',
+        'e2e': {'value': replicas.whole_job_rate(B * S, args.steps, e2e_ms), 'unit': 'tokens/s',
                 'h2d_bytes_per_step': h2d, 'd2h_bytes_per_step': d2h, 'ms_per_step': e2e_ms / args.steps},
         'gpu_launches': KERNELS_PER_STEP * args.steps,
         'clocks': clocks,
