@@ -78,7 +78,9 @@ typedef struct {
 /* Byte offsets of the regions inside the workspace that carries results from
  * transmla_mla_decode to transmla_mla_combine.  All regions are written by transmla_mla_decode.
  *   q_hat       bf16  [B, S, H, r+dR]   absorbed queries (Eq. 9 right, first line)
- *   cum_pages   int32 [B+1]             slot prefix sums: a sequence with n_b = ceil(L_b/P) > 0 pages owns
+ *   cum_pages   int32 [3B+1]            [0..B]: slot prefix sums (below); [B+1..3B]: per sequence the first and
+ *                                       last partition that holds pages of it (0, -1 for an empty sequence).
+ *                                       Prefix sums: a sequence with n_b = ceil(L_b/P) > 0 pages owns
  *                                       TRANSMLA_SEGMENT_COST_PAGES virtual slots followed by its n_b page
  *                                       slots; cum[b] = number of slots before sequence b
  *   plan        int32 [G, 4]            per partition: slot begin, end, sequence of first slot, sequence of

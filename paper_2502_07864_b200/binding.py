@@ -196,6 +196,7 @@ def workspace_views(params, workspace, lay=None):
     return {
         'q_hat': view(lay.q_hat_offset, B * SH * K, torch.bfloat16).view(B, params.q_len, params.num_heads, K),
         'cum_pages': view(lay.cum_pages_offset, B + 1, torch.int32),
+        'seq_parts': view(lay.cum_pages_offset, 3 * B + 1, torch.int32)[B + 1:].view(B, 2),
         'plan': view(lay.plan_offset, lay.num_partitions * 4, torch.int32).view(lay.num_partitions, 4),
         'partial_o': view(lay.partial_o_offset, lay.num_slots * SH * r, torch.float32).view(lay.num_slots, SH, r),
         'partial_lse': view(lay.partial_lse_offset, lay.num_slots * SH, torch.float32).view(lay.num_slots, SH),

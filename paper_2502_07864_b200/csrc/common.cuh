@@ -87,6 +87,22 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// Optional kernel-level timeline (compile with -DTRANSMLA_TRACE): global-timer time of the first block start
+// and the last block end of each kernel, to see how the step's kernels overlap in a pipelined run.
+#ifdef TRANSMLA_TRACE
+extern __device__ unsigned long long g_ktrace[8][2];
+__device__ __forceinline__ unsigned long long trace_now() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+#define TRK_BEGIN(k) do { if (threadIdx.x == 0) atomicMin(&g_ktrace[k][0], trace_now()); } while (0)
+#define TRK_END(k) do { if (threadIdx.x == 0) atomicMax(&g_ktrace[k][1], trace_now()); } while (0)
+#else
+#define TRK_BEGIN(k) do { } while (0)
+#define TRK_END(k) do { } while (0)
+#endif
+
 // Launchers (host).  Each enqueues on `stream` and returns the launch error, if any.
 cudaError_t launch_absorb_plan(const transmla_params_t& p, int G, const __nv_bfloat16* q_nope,
                                const __nv_bfloat16* q_pe, const __nv_bfloat16* w_uk, __nv_bfloat16* q_hat,

@@ -208,6 +208,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
   const int part = blockIdx.x, rb = blockIdx.y;
   const int SH = S * H;
   pdl_trigger();
+  TRK_BEGIN(1);
 
   if (tid == 0) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&cache_map)) : "memory");
@@ -529,6 +530,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
   }
 
   if (tid == 0) { TR(13, 1); TR_GLOBAL(10); }
+  TRK_END(1);
   // ---- teardown: everyone arrives, tensor memory is returned
   tc_fence_before();
   __syncthreads();

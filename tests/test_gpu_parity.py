@@ -36,6 +36,10 @@ def _run_and_compare(shape, seqlens, seed, G=0, scale=None, nan_tails=True, chec
         cum, plan = orc.split_plan(seqlens, shape.page_size, lay.num_partitions)
         assert np.array_equal(views['cum_pages'].cpu().numpy(), cum)
         assert np.array_equal(views['plan'].cpu().numpy(), plan)
+        want_parts = np.array([[0, -1]] * len(seqlens))
+        for (i, b, _, _, _) in orc.plan_segments(cum, plan):
+            want_parts[b] = (i, i) if want_parts[b][1] < 0 else (min(want_parts[b][0], i), max(want_parts[b][1], i))
+        assert np.array_equal(views['seq_parts'].cpu().numpy(), want_parts)
         # absorbed queries: bf16 rounding of an fp32 sum
         q_hat = orc.absorb(c['q_nope'], c['q_pe'], c['w_uk'])
         got = lifts.f64(views['q_hat'])
@@ -153,6 +157,10 @@ def test_combine_alone_on_oracle_partials():
     v = binding.workspace_views(params, ws, lay)
     cum, plan = orc.split_plan(seqlens, 64, G)
     v['cum_pages'].copy_(torch.tensor(cum))
+    parts = np.array([[0, -1]] * len(seqlens), dtype=np.int32)
+    for (i, b, _, _, _) in orc.plan_segments(cum, plan):
+        parts[b] = (i, i) if parts[b][1] < 0 else (min(parts[b][0], i), max(parts[b][1], i))
+    v['seq_parts'].copy_(torch.tensor(parts))
     v['partial_lse'].fill_(float('nan'))
     v['partial_o'].fill_(float('nan'))
     q_hat = orc.absorb(c['q_nope'], c['q_pe'], c['w_uk'])
