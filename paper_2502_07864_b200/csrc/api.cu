@@ -156,7 +156,6 @@ transmla_status_t transmla_mla_decode(const transmla_params_t* p, const void* q_
 transmla_status_t transmla_mla_combine(const transmla_params_t* p, const void* workspace, size_t workspace_bytes,
                                        const void* w_uv, void* out, float* lse_out, int32_t* dev_status,
                                        void* stream) {
-  (void)dev_status;
   transmla_workspace_layout_t lay;
   transmla_status_t st = transmla_workspace_layout(p, &lay);
   if (st != TRANSMLA_OK) return st;
@@ -171,7 +170,7 @@ transmla_status_t transmla_mla_combine(const transmla_params_t* p, const void* w
                                  reinterpret_cast<const float*>(ws + lay.partial_o_offset),
                                  reinterpret_cast<const float*>(ws + lay.partial_lse_offset),
                                  static_cast<const __nv_bfloat16*>(w_uv), static_cast<__nv_bfloat16*>(out), lse_out,
-                                 static_cast<cudaStream_t>(stream));
+                                 dev_status, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? TRANSMLA_OK : TRANSMLA_ERR_CUDA;
 }
 

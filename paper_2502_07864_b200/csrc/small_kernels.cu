@@ -395,153 +395,143 @@ cudaError_t launch_prologue(const transmla_params_t& p, int G, const __nv_bfloat
 }
 
 // ------------------------------------------------------------------------------------------------
-// Combine + up-projection (Eq. 9 right, last line before W_O).  Block = one head x ROWS query rows, 16 warps.
-// Phase 1: 16/ROWS warps share a row and merge its split partials by their lse (segments of sequence b live
-// in slots i + b for the partitions i of seq_parts[b]); the loads of up to 16 float4 per lane are in flight
-// together.  The merged row goes to shared memory as a bf16 hi/lo pair, in kperm order, so that the
-// tensor-core product of phase 2 carries fp32-like precision of o_hat.
-// Phase 2: out[rows, h, :] = o_hat W_UV_h^T, one 8-column output tile per warp with four independent
-// accumulator chains, W_UV_h read straight from global memory (pulled towards L2 before the dependency
-// wait), 16 bytes per lane.
+// Combine + up-projection (Eq. 9 right, last line before W_O).  Block = one head x 8 or 16 query rows
+// x (optionally) one half of the dv output columns.
+// Phase 1: each warp merges the split partials of its rows by their lse (segments of sequence b live
+// in slots i + b for the partitions i that overlap its pages) into shared memory as a bf16 hi/lo
+// pair, so that the tensor-core product of phase 2 carries fp32-like precision of o_hat.  The merged
+// row is stored in kperm order.
+// Phase 2: out[rows, h, :] = o_hat W_UV_h^T with W_UV_h read straight from global memory, 16 bytes per
+// lane and all loads of a tile in flight together.
 // ------------------------------------------------------------------------------------------------
-constexpr int kCombineThreads = 512;
+constexpr int kCombineRows = 16;
 
-template <int ROWS>
-__global__ void __launch_bounds__(kCombineThreads, 1)
-combine_kernel(const int32_t* __restrict__ cum, const float* __restrict__ partial_o,
-               const float* __restrict__ partial_lse, const __nv_bfloat16* __restrict__ w_uv,
-               __nv_bfloat16* __restrict__ out, float* __restrict__ lse_out, int B, int S, int H, int r, int dv, int G) {
-  constexpr int WPR = 16 / ROWS;   // warps that share a row in phase 1
-  constexpr int NC = 4 / WPR;      // float4 per lane and segment (r <= 512)
-  constexpr int SB = 16 / NC;      // segments per round
+__global__ void __launch_bounds__(256) combine_kernel(const int32_t* __restrict__ cum,
+                                                      const float* __restrict__ partial_o,
+                                                      const float* __restrict__ partial_lse,
+                                                      const __nv_bfloat16* __restrict__ w_uv,
+                                                      __nv_bfloat16* __restrict__ out, float* __restrict__ lse_out,
+                                                      int B, int S, int H, int r, int dv, int G, int rows_per_block) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int pitch = r + 8;
-  __nv_bfloat16* o_hi = reinterpret_cast<__nv_bfloat16*>(smem_raw);  // [16][pitch], rows ROWS..15 stay zero
-  __nv_bfloat16* o_lo = o_hi + 16 * pitch;                           // [16][pitch]
+  __nv_bfloat16* o_hi = reinterpret_cast<__nv_bfloat16*>(smem_raw);  // [16][pitch]
+  __nv_bfloat16* o_lo = o_hi + kCombineRows * pitch;                 // [16][pitch]
   pdl_trigger();
   TRK_BEGIN(2);
-  const int h = blockIdx.x, bs0 = blockIdx.y * ROWS;
+  const int h = blockIdx.x, bs0 = blockIdx.y * rows_per_block;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int SH = S * H, BS = B * S;
   const int g = lane >> 2, t4 = lane & 3, mi = lane >> 3;
-  const int tiles = dv / 8;
-  // weights do not depend on earlier kernels: pull this warp's rows of W_UV_h towards L2 now
-  for (int nt = warp; nt < tiles; nt += 16)
-    if (t4 == 0)
-      for (int k = 0; k < r; k += 64) prefetch_l2(w_uv + (static_cast<size_t>(h) * dv + nt * 8 + g) * r + k);
-  if (ROWS < 16) {
-    for (int i = tid; i < (16 - ROWS) * pitch / 8; i += kCombineThreads) {
-      reinterpret_cast<uint4*>(o_hi + ROWS * pitch)[i] = make_uint4(0, 0, 0, 0);
-      reinterpret_cast<uint4*>(o_lo + ROWS * pitch)[i] = make_uint4(0, 0, 0, 0);
-    }
-  }
-  pdl_wait();  // the partials, the slot prefix sums and the partition ranges come from the kernels before this one
-  TRC(0);
-
+  const int tiles = dv / 8, tiles_per_z = (tiles + gridDim.z - 1) / gridDim.z;
+  const int nt_lo = blockIdx.z * tiles_per_z, nt_hi = min(tiles, nt_lo + tiles_per_z);
+  // The weights do not depend on the merge: the first tile's 16-byte loads are issued now and land while
+  // the partials are merged.
+  constexpr int kWin = 16;  // windows of 32 columns held in registers (r <= 512 fits one round)
+  uint4 wv[kWin];
   {
-    const int rr = warp / WPR, sub = warp % WPR;
-    const int bs = bs0 + rr;
-    float acc[NC][4];
+    const int nt = nt_lo + warp;
+    const __nv_bfloat16* wrow = w_uv + (static_cast<size_t>(h) * dv + min(nt, tiles - 1) * 8 + g) * r + t4 * 8;
 #pragma unroll
-    for (int c = 0; c < NC; ++c) acc[c][0] = acc[c][1] = acc[c][2] = acc[c][3] = 0.f;
+    for (int u = 0; u < kWin; ++u) wv[u] = (nt < nt_hi && u * 32 < r) ? ld_u128(wrow + u * 32) : make_uint4(0, 0, 0, 0);
+  }
+  pdl_wait();  // the partials and the prefix sums come from the kernels before this one
+  const long long T = cum[B];
+
+  for (int rr = warp; rr < kCombineRows; rr += 8) {
+    const int bs = bs0 + rr;
+    float acc[4][4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) acc[c][0] = acc[c][1] = acc[c][2] = acc[c][3] = 0.f;
     float lse = -INFINITY, inv = 0.f;
-    if (bs < BS) {
+    if (rr < rows_per_block && bs < BS) {
       const int b = bs / S, s = bs % S, row = s * H + h;
       const int32_t* seq_parts = cum + B + 1;  // only 4-byte aligned: B + 1 may be odd
-      const int2 parts = make_int2(seq_parts[2 * b], seq_parts[2 * b + 1]);
-      const long long T = cum[B];
-      const int i_first = parts.x, nseg = parts.y - parts.x + 1;
-      if (T + nseg > 0) TRCK(8);
+      const int i_first = seq_parts[2 * b], nseg = seq_parts[2 * b + 1] - i_first + 1;
+      const bool dense = T >= G;  // then every partition owns at least one slot
       if (nseg > 0) {
-        const bool dense = T >= G;  // then every partition owns at least one slot
-        auto seg_exists = [&](int j) -> bool {  // candidate partition j of this sequence is not empty
-          if (j >= nseg) return false;
-          if (dense) return true;
+        auto seg_lse = [&](int j) -> float {  // lse of the j-th candidate partition, -inf if it is empty or absent
+          if (j >= nseg) return -INFINITY;
           const int pi = i_first + j;
-          return (static_cast<long long>(pi + 1) * T) / G > (static_cast<long long>(pi) * T) / G;
-        };
-        const size_t seg_stride = static_cast<size_t>(SH) * r;
-        const float* po0 = partial_o + (static_cast<size_t>(i_first + b) * SH + row) * r + sub * 128 + lane * 4;
-        const float* pl0 = partial_lse + static_cast<size_t>(i_first + b) * SH + row;
-        float4 v[SB][NC];
-        float l[SB];
-        auto load_batch = [&](int base) {
-#pragma unroll
-          for (int u = 0; u < SB; ++u) {
-            const bool ex = seg_exists(base + u);
-            l[u] = ex ? pl0[static_cast<size_t>(base + u) * SH] : -INFINITY;
-#pragma unroll
-            for (int c = 0; c < NC; ++c) {
-              v[u][c] = make_float4(0.f, 0.f, 0.f, 0.f);
-              if (ex && (c * WPR + sub) * 128 + lane * 4 < r)
-                v[u][c] = *reinterpret_cast<const float4*>(po0 + (base + u) * seg_stride + c * WPR * 128);
-            }
+          if (!dense) {
+            const long long p0 = (static_cast<long long>(pi) * T) / G, p1 = (static_cast<long long>(pi + 1) * T) / G;
+            if (p1 <= p0) return -INFINITY;
           }
+          return partial_lse[static_cast<size_t>(pi + b) * SH + row];
         };
-        load_batch(0);  // in flight while the maximum is found
         float m = -INFINITY;
-        for (int base = 0; base < nseg; base += 32)
-          m = fmaxf(m, seg_exists(base + lane) ? pl0[static_cast<size_t>(base + lane) * SH] : -INFINITY);
+        for (int base = 0; base < nseg; base += 32) m = fmaxf(m, seg_lse(base + lane));
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-        if (m > -1e30f) TRCK(9);
         if (m > -INFINITY) {
           float den = 0.f;
-          for (int base = 0; base < nseg; base += SB) {
-            if (base > 0) load_batch(base);
+          for (int base = 0; base < nseg; base += 32) {
+            const float l = seg_lse(base + lane);
+            const float wgt = l > -INFINITY ? __expf(l - m) : 0.f;
+            den += wgt;
+            const int cnt = min(32, nseg - base);
+            const float* po0 = partial_o + (static_cast<size_t>(i_first + base + b) * SH + row) * r + lane * 4;
+            const size_t seg_stride = static_cast<size_t>(SH) * r;
+            // four segments per round so that their loads overlap; a zero weight skips the (unwritten) slot
+            for (int j0 = 0; j0 < cnt; j0 += 4) {
+              float wj[4];
+              float4 v[4][4];
 #pragma unroll
-            for (int u = 0; u < SB; ++u) {
-              const float wj = l[u] > -INFINITY ? __expf(l[u] - m) : 0.f;  // an empty or all-masked segment weighs nothing
-              den += wj;
-              if (wj != 0.f) {
+              for (int u = 0; u < 4; ++u) {
+                wj[u] = (j0 + u < cnt) ? __shfl_sync(0xffffffffu, wgt, (j0 + u) & 31) : 0.f;
 #pragma unroll
-                for (int c = 0; c < NC; ++c) {
-                  acc[c][0] = fmaf(wj, v[u][c].x, acc[c][0]); acc[c][1] = fmaf(wj, v[u][c].y, acc[c][1]);
-                  acc[c][2] = fmaf(wj, v[u][c].z, acc[c][2]); acc[c][3] = fmaf(wj, v[u][c].w, acc[c][3]);
+                for (int c = 0; c < 4; ++c) {
+                  v[u][c] = make_float4(0.f, 0.f, 0.f, 0.f);
+                  if (wj[u] != 0.f && c * 128 + lane * 4 < r)
+                    v[u][c] = *reinterpret_cast<const float4*>(po0 + (j0 + u) * seg_stride + c * 128);
                 }
               }
+#pragma unroll
+              for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                  acc[c][0] = fmaf(wj[u], v[u][c].x, acc[c][0]); acc[c][1] = fmaf(wj[u], v[u][c].y, acc[c][1]);
+                  acc[c][2] = fmaf(wj[u], v[u][c].z, acc[c][2]); acc[c][3] = fmaf(wj[u], v[u][c].w, acc[c][3]);
+                }
             }
           }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
           inv = 1.f / den;
           lse = m + __logf(den);
-          if (inv > 0.f) TRCK(10);
         }
       }
-      if (lse_out != nullptr && lane == 0 && sub == 0) lse_out[(static_cast<size_t>(b) * S + s) * H + h] = lse;
+      if (lse_out != nullptr && lane == 0 && blockIdx.z == 0) lse_out[(static_cast<size_t>(b) * S + s) * H + h] = lse;
     }
 #pragma unroll
-    for (int c = 0; c < NC; ++c) {
-      const int k = (c * WPR + sub) * 128 + lane * 4;
+    for (int c = 0; c < 4; ++c) {
+      const int k = c * 128 + lane * 4;
       if (k < r) {
-        float vv[4], lo[4];
+        float v[4], lo[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          vv[e] = acc[c][e] * inv;
-          lo[e] = vv[e] - __bfloat162float(__float2bfloat16_rn(vv[e]));
+          v[e] = acc[c][e] * inv;
+          lo[e] = v[e] - __bfloat162float(__float2bfloat16_rn(v[e]));
         }
         const int win = k & ~31, p = k & 31;  // elements p..p+3 of the window: two pairs, each stays adjacent
         const int q0 = win + kperm(p), q1 = win + kperm(p + 2);
-        *reinterpret_cast<uint32_t*>(o_hi + rr * pitch + q0) = pack_bf16(vv[0], vv[1]);
-        *reinterpret_cast<uint32_t*>(o_hi + rr * pitch + q1) = pack_bf16(vv[2], vv[3]);
+        *reinterpret_cast<uint32_t*>(o_hi + rr * pitch + q0) = pack_bf16(v[0], v[1]);
+        *reinterpret_cast<uint32_t*>(o_hi + rr * pitch + q1) = pack_bf16(v[2], v[3]);
         *reinterpret_cast<uint32_t*>(o_lo + rr * pitch + q0) = pack_bf16(lo[0], lo[1]);
         *reinterpret_cast<uint32_t*>(o_lo + rr * pitch + q1) = pack_bf16(lo[2], lo[3]);
       }
     }
   }
-  TRC(1);
   __syncthreads();
-  TRC(2);
 
-  constexpr int kWin = 16;  // windows of 32 columns whose weight loads are in flight together
-  for (int nt = warp; nt < tiles; nt += 16) {
-    float acc[4][4];  // hi/lo x even/odd k-step: four independent chains, summed at the end
-#pragma unroll
-    for (int q = 0; q < 4; ++q) acc[q][0] = acc[q][1] = acc[q][2] = acc[q][3] = 0.f;
+  for (int nt = nt_lo + warp; nt < nt_hi; nt += 8) {
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
     const __nv_bfloat16* wrow = w_uv + (static_cast<size_t>(h) * dv + nt * 8 + g) * r + t4 * 8;
-    for (int w0 = 0; w0 < r; w0 += kWin * 32) {
-      uint4 wv[kWin];
+    for (int w0 = 0; w0 < r; w0 += kWin * 32) {  // kWin windows per round, all their loads in flight together
+      if (nt != nt_lo + warp || w0 != 0) {
 #pragma unroll
-      for (int u = 0; u < kWin; ++u) wv[u] = (w0 + u * 32 < r) ? ld_u128(wrow + w0 + u * 32) : make_uint4(0, 0, 0, 0);
+        for (int u = 0; u < kWin; ++u)
+          wv[u] = (w0 + u * 32 < r) ? ld_u128(wrow + w0 + u * 32) : make_uint4(0, 0, 0, 0);
+      }
 #pragma unroll
       for (int u = 0; u < kWin; ++u) {
         if (w0 + u * 32 < r) {
@@ -549,42 +539,35 @@ combine_kernel(const int32_t* __restrict__ cum, const float* __restrict__ partia
           const int off = ((mi & 1) * 8 + (lane & 7)) * pitch + w0 + u * 32 + (mi >> 1) * 8;
           ldmatrix_x4(ah, o_hi + off);
           ldmatrix_x4(al, o_lo + off);
-          mma_bf16_16816(acc[0], ah, wv[u].x, wv[u].y);
-          mma_bf16_16816(acc[1], al, wv[u].x, wv[u].y);
+          mma_bf16_16816(acc, ah, wv[u].x, wv[u].y);
+          mma_bf16_16816(acc, al, wv[u].x, wv[u].y);
           ldmatrix_x4(ah, o_hi + off + 16);
           ldmatrix_x4(al, o_lo + off + 16);
-          mma_bf16_16816(acc[2], ah, wv[u].z, wv[u].w);
-          mma_bf16_16816(acc[3], al, wv[u].z, wv[u].w);
+          mma_bf16_16816(acc, ah, wv[u].z, wv[u].w);
+          mma_bf16_16816(acc, al, wv[u].z, wv[u].w);
         }
       }
     }
-    const float o0 = (acc[0][0] + acc[2][0]) + (acc[1][0] + acc[3][0]), o1 = (acc[0][1] + acc[2][1]) + (acc[1][1] + acc[3][1]);
-    const float o2 = (acc[0][2] + acc[2][2]) + (acc[1][2] + acc[3][2]), o3 = (acc[0][3] + acc[2][3]) + (acc[1][3] + acc[3][3]);
+    const int col = nt * 8 + t4 * 2;
     const int bs_a = bs0 + g, bs_b = bs0 + g + 8;
-    if (g < ROWS && bs_a < BS)
-      *reinterpret_cast<uint32_t*>(out + (static_cast<size_t>(bs_a) * H + h) * dv + nt * 8 + t4 * 2) = pack_bf16(o0, o1);
-    if (g + 8 < ROWS && bs_b < BS)
-      *reinterpret_cast<uint32_t*>(out + (static_cast<size_t>(bs_b) * H + h) * dv + nt * 8 + t4 * 2) = pack_bf16(o2, o3);
+    if (g < rows_per_block && bs_a < BS)
+      *reinterpret_cast<uint32_t*>(out + (static_cast<size_t>(bs_a) * H + h) * dv + col) = pack_bf16(acc[0], acc[1]);
+    if (g + 8 < rows_per_block && bs_b < BS)
+      *reinterpret_cast<uint32_t*>(out + (static_cast<size_t>(bs_b) * H + h) * dv + col) = pack_bf16(acc[2], acc[3]);
   }
-  TRK_END(2);
-  TRC(3);
 }
 
 cudaError_t launch_combine(const transmla_params_t& p, int G, const int32_t* cum, const float* partial_o,
                            const float* partial_lse, const __nv_bfloat16* w_uv, __nv_bfloat16* out, float* lse_out,
-                           cudaStream_t stream) {
+                           int32_t* dev_status, cudaStream_t stream) {
+  (void)dev_status;
   const int BS = p.batch * p.q_len;
-  const size_t smem = 2 * 16 * (p.kv_lora_rank + 8) * sizeof(__nv_bfloat16);
-  auto go = [&](auto kernel, int rows) {
-    dim3 grid(p.num_heads, (BS + rows - 1) / rows);
-    return launch_pdl(kernel, grid, dim3(kCombineThreads), smem, stream, cum, partial_o, partial_lse, w_uv, out, lse_out,
-                      p.batch, p.q_len, p.num_heads, p.kv_lora_rank, p.v_dim, G);
-  };
-  // few query rows: small row blocks so that the grid still covers the SMs; many: full 16-row tiles
-  const int blocks4 = p.num_heads * ((BS + 3) / 4);
-  if (blocks4 <= 160) return go(combine_kernel<4>, 4);
-  if (blocks4 <= 640) return go(combine_kernel<8>, 8);
-  return go(combine_kernel<16>, 16);
+  const int rows = BS <= 64 ? 8 : 16;  // smaller blocks when there are few query rows, for more parallelism
+  const int zsplit = (BS <= 64 && p.v_dim >= 128) ? 2 : 1;
+  dim3 grid(p.num_heads, (BS + rows - 1) / rows, zsplit);
+  const size_t smem = 2 * kCombineRows * (p.kv_lora_rank + 8) * sizeof(__nv_bfloat16);
+  return launch_pdl(combine_kernel, grid, dim3(256), smem, stream, cum, partial_o, partial_lse, w_uv, out, lse_out,
+                    p.batch, p.q_len, p.num_heads, p.kv_lora_rank, p.v_dim, G, rows);
 }
 
 }  // namespace transmla
