@@ -67,7 +67,8 @@ typedef struct {
   int32_t num_pages;         /* pages in the cache pool */
   int32_t max_pages_per_seq; /* row stride of page_table */
   int32_t batch;             /* B */
-  int32_t num_partitions;    /* G: how many pieces the batch's pages are split into; 0 = library chooses */
+  int32_t num_partitions;    /* G: how many pieces the batch's pages are split into; 0 = library chooses
+                                (SMs / row blocks, at most batch * max_pages_per_seq / 4) */
   float softmax_scale;       /* 1/sqrt(dn + dR) for MLA (Eq. 9), 1/sqrt(d) for a lifted GQA layer (Eq. 13) */
   float rope_theta;          /* RoPE base, 10000 in Eq. 1 */
 } transmla_params_t;

@@ -66,6 +66,10 @@ transmla_status_t transmla_workspace_layout(const transmla_params_t* p, transmla
     if (st != TRANSMLA_OK) return st;
     const int row_blocks = (p->q_len * p->num_heads + kRowBlock - 1) / kRowBlock;
     G = sms / row_blocks;
+    // Small problems: no more partitions than a quarter of the pages the batch can hold, so that a partition
+    // keeps at least about four pages and a sequence is not cut into dozens of one-page partials.
+    const long long cap = (static_cast<long long>(p->batch) * p->max_pages_per_seq + 3) / 4;
+    if (G > cap) G = static_cast<int>(cap);
     if (G < 1) G = 1;
   }
   const size_t B = p->batch, SH = static_cast<size_t>(p->q_len) * p->num_heads;
