@@ -70,6 +70,20 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
       : "memory");
 }
+// The same with an L2 eviction hint.  Cache pages are read once per step: marking them evict-first keeps the
+// few MB of weights and split partials that the neighbouring kernels reuse resident in L2.
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+  uint64_t policy;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+  return policy;
+}
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar,
+                                                 uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar), "l"(policy)
+      : "memory");
+}
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -200,6 +214,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
       // ======================================================================== TMA producer
       // The ring carries, per segment, one item with the 32 absorbed query rows followed by the segment's pages.
       int g = 0;  // ring items issued by this CTA so far
+      const uint64_t stream_policy = l2_evict_first_policy();
       auto acquire = [&](int gi) -> uint32_t {  // waits for the stage of ring item gi; returns its index
         const int stage = gi % kStages, use = gi / kStages;
         mbar_wait(bar(BAR_KV_EMPTY + stage), (use & 1) ^ 1, abort_flag, dev_status);
@@ -231,7 +246,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
             const uint32_t dst = base + kOffStage + stage * kStageBytes;
 #pragma unroll
             for (int c = 0; c < kChunks; ++c)
-              tma_load_2d(dst + c * kSubTileBytes, &cache_map, c * 64, idx * kPage, bar(BAR_KV_FULL + stage));
+              tma_load_2d_hint(dst + c * kSubTileBytes, &cache_map, c * 64, idx * kPage, bar(BAR_KV_FULL + stage), stream_policy);
           }
           __syncwarp();
         }
