@@ -187,6 +187,12 @@ def run_ours(args, name, shape, seqlens, seed):
     dc = synth.make_decode_case(shape, seqlens, replicas.rank_seed(seed, rank), device='cuda')
     ac = synth.make_append_case(shape, [L - S for L in seqlens], replicas.rank_seed(seed, rank) + 1, device='cuda')
     caches = [dc['cache']] + [dc['cache'].clone() for _ in range(n_copies - 1)]
+    # Weights rotate as well (their copies together exceed L2): in a whole model every other layer's weights pass
+    # through L2 between two steps of this layer, so a step must find its own weights in HBM, not in L2.
+    n_w = args.weight_copies
+    weights = [(ac['w_dkv_kr'], dc['w_uk'], dc['w_uv'])] + [
+        (ac['w_dkv_kr'].clone(), dc['w_uk'].clone(), dc['w_uv'].clone()) for _ in range(n_w - 1)]
+    weight_bytes = sum(t.numel() * t.element_size() for t in weights[0])
     params = binding.make_params(shape, B, dc['cache'].shape[0], dc['page_table'].shape[1], scale)
     ws, lay = binding.alloc_workspace(params)
     out = torch.empty(B, S, H, shape.dv, dtype=torch.bfloat16, device='cuda')
@@ -198,7 +204,7 @@ def run_ours(args, name, shape, seqlens, seed):
         if ev is not None:
             binding.transmla_profile_decode_kernel(ev[0], ev[1])
         binding.transmla_decode_step(params, ac['x'], dc['q_nope'], dc['q_pe'], dc['page_table'], dc['seqlens'],
-                                     ac['w_dkv_kr'], dc['w_uk'], dc['w_uv'], caches[i % n_copies], ws, out, lse,
+                                     *weights[i % n_w], caches[i % n_copies], ws, out, lse,
                                      status, stream)
 
     def barrier():
@@ -239,7 +245,7 @@ def run_ours(args, name, shape, seqlens, seed):
 
     def host_step(i):
         return binding.transmla_decode_step_host(params, h['x'], h['q_nope'], h['q_pe'], h['page_table'], h['seqlens'],
-                                                 ac['w_dkv_kr'], dc['w_uk'], dc['w_uv'], caches[i % n_copies], staging,
+                                                 *weights[i % n_w], caches[i % n_copies], staging,
                                                  ws, h_out, h_lse, stream)
     for i in range(3):
         host_step(i)
@@ -273,7 +279,8 @@ def run_ours(args, name, shape, seqlens, seed):
         'config': {'workload': name, 'batch_per_gpu': B, 'q_len': S, 'heads': H, 'latent': shape.r, 'rope': shape.dR,
                    'cached_tokens_per_gpu': sum(seqlens), 'page_size': shape.page_size,
                    'num_partitions': lay.num_partitions,
-                   'l2': f'cache rotates over {n_copies} copies ({n_copies * cache_bytes / 1e6:.0f} MB) between steps',
+                   'l2': f'cache rotates over {n_copies} copies ({n_copies * cache_bytes / 1e6:.0f} MB) and the weights '
+                         f'over {n_w} copies ({n_w * weight_bytes / 1e6:.0f} MB) between steps',
                    'parallelism': f'replicas x{world}, no data-path collective'},
         'cache_gbs': world * cache_bytes / (ms_step * 1e-3) / 1e9,
         'cache_gbs_pct_of_8tbs': 100.0 * cache_bytes / (ms_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
@@ -301,6 +308,7 @@ def main():
     ap.add_argument('--impl', default='ours', choices=['ours', 'reference'])
     ap.add_argument('--workload', default='llama2-7b-mla_b16_8k')
     ap.add_argument('--cache-copies', type=int, default=4)
+    ap.add_argument('--weight-copies', type=int, default=12)
     ap.add_argument('--no-cpu-baseline', action='store_true')
     args = ap.parse_args()
     w = workloads()
