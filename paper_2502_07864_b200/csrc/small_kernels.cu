@@ -555,6 +555,7 @@ __global__ void __launch_bounds__(256) combine_kernel(const int32_t* __restrict_
     if (g + 8 < rows_per_block && bs_b < BS)
       *reinterpret_cast<uint32_t*>(out + (static_cast<size_t>(bs_b) * H + h) * dv + col) = pack_bf16(acc[2], acc[3]);
   }
+  TRK_END(2);
 }
 
 cudaError_t launch_combine(const transmla_params_t& p, int G, const int32_t* cum, const float* partial_o,
