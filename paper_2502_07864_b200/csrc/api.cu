@@ -1,6 +1,5 @@
 // C ABI of the absorbed-MLA decode library: argument checks, workspace layout, launches.
 #include <cstdio>
-#include <cstdlib>
 #include <cstring>
 #include <unordered_set>
 #include <vector>
@@ -126,8 +125,7 @@ static transmla_status_t launch_split_kv(const transmla_params_t* p, const trans
   cudaEvent_t ev0 = tl_prof_start, ev1 = tl_prof_stop;
   tl_prof_start = tl_prof_stop = nullptr;
   if (ev0 != nullptr && cudaEventRecord(ev0, s) != cudaSuccess) return TRANSMLA_ERR_CUDA;
-  static const bool force_generic = getenv("TRANSMLA_FORCE_GENERIC") != nullptr;
-  auto launch = (decode_sm100_supported(*p) && !force_generic) ? launch_decode_sm100 : launch_decode_generic;
+  auto launch = decode_sm100_supported(*p) ? launch_decode_sm100 : launch_decode_generic;
   if (launch(*p, lay.num_partitions, reinterpret_cast<__nv_bfloat16*>(ws + lay.q_hat_offset),
              static_cast<const __nv_bfloat16*>(cache), page_table, seqlens,
              reinterpret_cast<int32_t*>(ws + lay.cum_pages_offset), reinterpret_cast<int32_t*>(ws + lay.plan_offset),

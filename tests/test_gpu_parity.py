@@ -96,6 +96,30 @@ def test_llama_shape_medium(seqlens, G):
     _run_and_compare(synth.LLAMA2_7B, seqlens, seed=2, G=G, check_internals=(len(seqlens) == 3 and G == 0))
 
 
+@pytest.mark.parametrize('H,S', [(8, 1), (40, 1), (24, 2)])
+def test_production_latent_with_row_counts_that_do_not_fill_a_block(H, S):
+    # r = 512, dR = 64 goes through the TMA/tcgen05 kernel; S*H = 8, 40, 48 leave the last 32-row block ragged
+    shape = synth.MLAShape(H=H, dn=128, dR=64, dv=128, r=512, D=4096, S=S)
+    _run_and_compare(shape, [300, 64, 2, 1100], seed=17, G=5, check_internals=True)
+
+
+def test_wide_heads_and_many_sequences():
+    # dn = dv = 256 (largest supported head dims) on the small latent; 5000 one-page sequences make the plan
+    # block take its global-memory path (more sequences than its shared-memory buffer holds)
+    shape = synth.MLAShape(H=4, dn=256, dR=16, dv=256, r=64, D=256)
+    _run_and_compare(shape, [70, 5, 129], seed=18, G=3)
+    many = [1 + (i * 7) % 60 for i in range(5000)]
+    case = synth.make_decode_case(synth.TINY, many, seed=19)
+    out, lse, status, views, lay = gu.gpu_decode(synth.TINY, gu.to_dev(case), gu.mla_scale(synth.TINY), G=0, want_views=True)
+    assert status == 0
+    cum, plan = orc.split_plan(many, 64, lay.num_partitions)
+    assert np.array_equal(views['cum_pages'].cpu().numpy(), cum) and np.array_equal(views['plan'].cpu().numpy(), plan)
+    only = [(b, 0, h) for b in (0, 1, 2499, 4999) for h in (0, 7)]
+    want, want_lse = gu.oracle_decode(synth.TINY, case, gu.mla_scale(synth.TINY), only=only)
+    idx = tuple(np.array(only).T)
+    gu.assert_close(lifts.f64(out)[idx], want[idx], 'many sequences')
+
+
 def test_qwen_shape_two_query_positions():
     shape = synth.QWEN25_72B
     _run_and_compare(shape, [130, 300, 2], seed=5, G=6, check_internals=True)
