@@ -228,6 +228,13 @@ transmla_status_t transmla_mla_attention_static(const transmla_params_t* params 
                                                 const int32_t* seqlens, void* out, float* lse_out,
                                                 int32_t* dev_status, void* stream);
 
+/* Diagnostic: demonstrates the bounded waits of the kernels (no counterpart in the paper).  Launches one
+ * block that waits, through the same helper the split-KV kernel uses, on a barrier that is never
+ * satisfied.  After the limit (about 0.2 s) the wait gives up, TRANSMLA_DEV_TIMEOUT is set in *dev_status
+ * (device int32, required), a second wait returns immediately and the kernel ends; the context stays
+ * usable.  cycles_out (device int64[2], may be NULL) receives the SM cycles spent in the two waits. */
+transmla_status_t transmla_selftest_bounded_wait(int32_t* dev_status, long long* cycles_out, void* stream);
+
 /* Timing hook: the next transmla_mla_decode issued by the calling thread records `start_event`
  * immediately before and `stop_event` immediately after its split-KV kernel on that call's stream
  * (both cudaEvent_t passed as void*; NULL, NULL clears the hook).  The hook is consumed by that call. */

@@ -14,7 +14,7 @@ _LIB_PATH = os.path.join(_HERE, 'libtransmla.so')
 EXPORTS = ('transmla_workspace_layout', 'transmla_latent_append', 'transmla_mla_decode', 'transmla_mla_combine',
            'transmla_validate_tables', 'transmla_step_staging_bytes', 'transmla_decode_step_host',
            'transmla_decode_step', 'transmla_profile_decode_kernel', 'transmla_status_string',
-           'transmla_static_workspace_capacity', 'transmla_mla_attention_static')
+           'transmla_static_workspace_capacity', 'transmla_mla_attention_static', 'transmla_selftest_bounded_wait')
 
 
 class Params(ctypes.Structure):
@@ -64,6 +64,7 @@ def lib():
         L.transmla_static_workspace_capacity.argtypes = []
         L.transmla_static_workspace_capacity.restype = sz
         L.transmla_mla_attention_static.argtypes = [pp, vp, vp, vp, vp, vp, i32p, i32p, vp, vp, i32p, vp]
+        L.transmla_selftest_bounded_wait.argtypes = [i32p, vp, vp]
         L.transmla_status_string.argtypes = [ctypes.c_int]
         L.transmla_status_string.restype = ctypes.c_char_p
         for name in EXPORTS:
@@ -169,6 +170,11 @@ def transmla_mla_attention_static(params, q_nope, q_pe, w_uk, w_uv, cache, page_
     _check(lib().transmla_mla_attention_static(
         ctypes.byref(params), _ptr(q_nope), _ptr(q_pe), _ptr(w_uk), _ptr(w_uv), _ptr(cache), _ptr(page_table),
         _ptr(seqlens), _ptr(out), _ptr(lse_out), _ptr(dev_status), _stream(stream)), 'transmla_mla_attention_static')
+
+
+def transmla_selftest_bounded_wait(dev_status, cycles_out=None, stream=None):
+    _check(lib().transmla_selftest_bounded_wait(_ptr(dev_status), _ptr(cycles_out), _stream(stream)),
+           'transmla_selftest_bounded_wait')
 
 
 def transmla_profile_decode_kernel(start_event, stop_event):

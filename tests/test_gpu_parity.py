@@ -203,6 +203,22 @@ def test_combine_alone_on_oracle_partials():
     gu.assert_lse_close(lifts.f64(lse), want_lse, 'combine lse')
 
 
+def test_a_wait_that_nothing_satisfies_ends_by_itself_and_leaves_the_context_usable():
+    import time
+    status = torch.zeros(1, dtype=torch.int32, device='cuda')
+    cycles = torch.zeros(2, dtype=torch.int64, device='cuda')
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    binding.transmla_selftest_bounded_wait(status, cycles)
+    torch.cuda.synchronize()
+    took = time.perf_counter() - t0
+    assert int(status.item()) & 2                    # TRANSMLA_DEV_TIMEOUT
+    assert 0.05 < took < 2.0
+    first, second = (int(v) for v in cycles.tolist())
+    assert first > 100_000_000 and second < 100_000  # the second wait does not spin again
+    _run_and_compare(synth.TINY, [17, 64], seed=1, G=2)   # and ordinary work still runs afterwards
+
+
 # ------------------------------------------------------------------ append
 @pytest.mark.parametrize('shape,positions', [(synth.TINY, [16, 63, 64, 0]), (synth.LLAMA2_7B, [8191, 0, 77, 131071]),
                                              (synth.QWEN25_72B, [126, 63, 4000])])
