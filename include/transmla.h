@@ -182,8 +182,10 @@ size_t transmla_step_staging_bytes(const transmla_params_t* params /* host */);
 /* One whole decode step driven from host buffers: validates the tables on the host, copies this
  * step's inputs to the device (x, q_nope, q_pe, page_table, seqlens), runs transmla_decode_step,
  * copies `out` (and `lse` if not NULL) back and waits for `stream`.  Weights and the cache stay
- * resident on the device.  Host buffers should be pinned for the copies to be asynchronous.  Uses
- * host heap memory for the validation; allocates no device memory.  Returns the first error, or
+ * resident on the device.  When the host arrays are pinned (page-locked) the transfers are done by one
+ * kernel each way that reads or writes the pinned memory directly; otherwise by one cudaMemcpyAsync per
+ * array.  Uses host heap memory for the validation and, once per calling thread, 64 bytes of pinned host
+ * memory for the status word; allocates no device memory.  Returns the first error, or
  * TRANSMLA_OK; `*h_dev_status` (host, may be NULL) receives the device status word.
  *   h_x [B,S,D], h_q_nope [B,S,H,dn], h_q_pe [B,S,H,dR], h_page_table, h_seqlens : host
  *   w_dkv_kr, w_uk, w_uv, cache, staging, workspace                              : device

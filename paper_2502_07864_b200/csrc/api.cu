@@ -45,6 +45,44 @@ transmla_status_t check_device(int* sm_count) {
 
 thread_local cudaEvent_t tl_prof_start = nullptr, tl_prof_stop = nullptr;
 
+// ---- host <-> device transfers of the host-buffer step done by one kernel each way.
+// Pinned host memory is addressable from the device, so a single launch can move all five input arrays (and
+// another one the results) instead of one copy-engine operation per array, each with its own start-up latency.
+struct CopyJob { const void* src; void* dst; unsigned long long bytes; };
+struct CopyList { CopyJob job[6]; int n; int32_t* zero_word; };
+
+__global__ void __launch_bounds__(256) copy_list_kernel(CopyList list) {
+  if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0 && list.zero_word != nullptr) *list.zero_word = 0;
+  if (static_cast<int>(blockIdx.y) >= list.n) return;
+  const CopyJob j = list.job[blockIdx.y];
+  const size_t tid = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x, nthr = static_cast<size_t>(gridDim.x) * blockDim.x;
+  if (((reinterpret_cast<uintptr_t>(j.src) | reinterpret_cast<uintptr_t>(j.dst) | j.bytes) & 15) == 0) {
+    const uint4* s = static_cast<const uint4*>(j.src);
+    uint4* d = static_cast<uint4*>(j.dst);
+    for (size_t i = tid; i < j.bytes / 16; i += nthr) d[i] = s[i];
+  } else {  // every array of the step is a whole number of 4-byte words
+    const uint32_t* s = static_cast<const uint32_t*>(j.src);
+    uint32_t* d = static_cast<uint32_t*>(j.dst);
+    for (size_t i = tid; i < j.bytes / 4; i += nthr) d[i] = s[i];
+  }
+}
+
+bool is_pinned_host(const void* p) {
+  cudaPointerAttributes a;
+  if (cudaPointerGetAttributes(&a, p) != cudaSuccess) { cudaGetLastError(); return false; }
+  return a.type == cudaMemoryTypeHost && (reinterpret_cast<uintptr_t>(p) & 3) == 0;
+}
+
+// One pinned word per calling thread for reading the device status back without a copy-engine operation.
+int32_t* pinned_status_word() {
+  thread_local int32_t* word = nullptr;
+  if (word == nullptr && cudaHostAlloc(reinterpret_cast<void**>(&word), 64, cudaHostAllocPortable) != cudaSuccess) {
+    cudaGetLastError();
+    word = nullptr;
+  }
+  return word;
+}
+
 }  // namespace
 
 extern "C" {
@@ -272,23 +310,49 @@ transmla_status_t transmla_decode_step_host(const transmla_params_t* p, const vo
 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   bool ok = true;
-  ok &= cudaMemcpyAsync(d_x, h_x, nx, cudaMemcpyHostToDevice, s) == cudaSuccess;
-  ok &= cudaMemcpyAsync(d_qn, h_q_nope, nqn, cudaMemcpyHostToDevice, s) == cudaSuccess;
-  if (nqp) ok &= cudaMemcpyAsync(d_qp, h_q_pe, nqp, cudaMemcpyHostToDevice, s) == cudaSuccess;
-  ok &= cudaMemcpyAsync(d_pt, h_page_table, npt, cudaMemcpyHostToDevice, s) == cudaSuccess;
-  ok &= cudaMemcpyAsync(d_sl, h_seqlens, B * 4, cudaMemcpyHostToDevice, s) == cudaSuccess;
-  ok &= cudaMemsetAsync(d_st, 0, 4, s) == cudaSuccess;
+  const bool in_pinned = is_pinned_host(h_x) && is_pinned_host(h_q_nope) && (nqp == 0 || is_pinned_host(h_q_pe)) &&
+                         is_pinned_host(h_page_table) && is_pinned_host(h_seqlens);
+  if (in_pinned) {
+    CopyList l = {};
+    l.job[l.n++] = {h_x, d_x, nx};
+    l.job[l.n++] = {h_q_nope, d_qn, nqn};
+    if (nqp) l.job[l.n++] = {h_q_pe, d_qp, nqp};
+    l.job[l.n++] = {h_page_table, d_pt, npt};
+    l.job[l.n++] = {h_seqlens, d_sl, B * 4};
+    l.zero_word = reinterpret_cast<int32_t*>(d_st);
+    copy_list_kernel<<<dim3(24, l.n), 256, 0, s>>>(l);
+    ok &= cudaGetLastError() == cudaSuccess;
+  } else {
+    ok &= cudaMemcpyAsync(d_x, h_x, nx, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    ok &= cudaMemcpyAsync(d_qn, h_q_nope, nqn, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    if (nqp) ok &= cudaMemcpyAsync(d_qp, h_q_pe, nqp, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    ok &= cudaMemcpyAsync(d_pt, h_page_table, npt, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    ok &= cudaMemcpyAsync(d_sl, h_seqlens, B * 4, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    ok &= cudaMemsetAsync(d_st, 0, 4, s) == cudaSuccess;
+  }
   if (!ok) return TRANSMLA_ERR_CUDA;
   auto* dst = reinterpret_cast<int32_t*>(d_st);
   st = transmla_decode_step(p, d_x, d_qn, d_qp, reinterpret_cast<int32_t*>(d_pt), reinterpret_cast<int32_t*>(d_sl),
                             w_dkv_kr, w_uk, w_uv, cache, workspace, workspace_bytes,
                             d_out, reinterpret_cast<float*>(d_lse), dst, stream);
   if (st != TRANSMLA_OK) return st;
-  ok &= cudaMemcpyAsync(h_out, d_out, nout, cudaMemcpyDeviceToHost, s) == cudaSuccess;
-  if (h_lse) ok &= cudaMemcpyAsync(h_lse, d_lse, nlse, cudaMemcpyDeviceToHost, s) == cudaSuccess;
   int32_t dev_word = 0;
-  ok &= cudaMemcpyAsync(&dev_word, d_st, 4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
-  ok &= cudaStreamSynchronize(s) == cudaSuccess;
+  int32_t* pinned_word = pinned_status_word();
+  if (pinned_word != nullptr && is_pinned_host(h_out) && (h_lse == nullptr || is_pinned_host(h_lse))) {
+    CopyList l = {};
+    l.job[l.n++] = {d_out, h_out, nout};
+    if (h_lse) l.job[l.n++] = {d_lse, h_lse, nlse};
+    l.job[l.n++] = {d_st, pinned_word, 4};
+    copy_list_kernel<<<dim3(24, l.n), 256, 0, s>>>(l);
+    ok &= cudaGetLastError() == cudaSuccess;
+    ok &= cudaStreamSynchronize(s) == cudaSuccess;
+    dev_word = *pinned_word;
+  } else {
+    ok &= cudaMemcpyAsync(h_out, d_out, nout, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+    if (h_lse) ok &= cudaMemcpyAsync(h_lse, d_lse, nlse, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+    ok &= cudaMemcpyAsync(&dev_word, d_st, 4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+    ok &= cudaStreamSynchronize(s) == cudaSuccess;
+  }
   if (h_dev_status) *h_dev_status = dev_word;
   return ok ? TRANSMLA_OK : TRANSMLA_ERR_CUDA;
 }

@@ -253,7 +253,8 @@ def test_append_values_slots_and_untouched_bytes(shape, positions):
 
 
 # ------------------------------------------------------------------ whole step from host buffers
-def test_decode_step_from_host_buffers():
+@pytest.mark.parametrize('pinned', [True, False])
+def test_decode_step_from_host_buffers(pinned):
     shape = synth.LLAMA2_7B
     seqlens = [300, 65, 1024]
     B = len(seqlens)
@@ -263,9 +264,10 @@ def test_decode_step_from_host_buffers():
     params = binding.make_params(shape, B, dc['cache'].shape[0], dc['page_table'].shape[1], scale)
     ws, _ = binding.alloc_workspace(params)
     staging = torch.empty(binding.transmla_step_staging_bytes(params), dtype=torch.uint8, device='cuda')
-    pin = lambda t: t.contiguous().pin_memory()
-    h_out = torch.empty(B, 1, shape.H, shape.dv, dtype=torch.bfloat16).pin_memory()
-    h_lse = torch.empty(B, 1, shape.H, dtype=torch.float32).pin_memory()
+    # pinned arrays go through the library's transfer kernels, pageable ones through cudaMemcpyAsync
+    pin = (lambda t: t.contiguous().pin_memory()) if pinned else (lambda t: t.contiguous().clone())
+    h_out = pin(torch.empty(B, 1, shape.H, shape.dv, dtype=torch.bfloat16))
+    h_lse = pin(torch.empty(B, 1, shape.H, dtype=torch.float32))
     cache = dc['cache'].cuda()
     word = binding.transmla_decode_step_host(params, pin(ac['x']), pin(dc['q_nope']), pin(dc['q_pe']),
                                              pin(dc['page_table']), pin(dc['seqlens']), ac['w_dkv_kr'].cuda(),
