@@ -487,13 +487,19 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
         tc_fence_after();
         float* dst = partial_o + (static_cast<size_t>(slot) * SH + rb * kRowBlock) * R + warp * 32 + lane;
 #pragma unroll 1
-        for (int t = 0; t < 4; ++t) {
-          uint32_t ov[32];
+        for (int t = 0; t < 4; t += 2) {  // two 128-row tiles per round trip to tensor memory
+          uint32_t ov[64];
           tmem_ld32(tmem + lane_base + kColO + t * 32, ov);
+          tmem_ld32(tmem + lane_base + kColO + (t + 1) * 32, ov + 32);
           tc_wait_ld();
 #pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (rb * kRowBlock + j < SH) dst[static_cast<size_t>(j) * R + t * 128] = __uint_as_float(ov[j]) * inv_l[j];
+          for (int j = 0; j < 32; ++j) {
+            if (rb * kRowBlock + j < SH) {
+              const float sc = inv_l[j];
+              dst[static_cast<size_t>(j) * R + t * 128] = __uint_as_float(ov[j]) * sc;
+              dst[static_cast<size_t>(j) * R + (t + 1) * 128] = __uint_as_float(ov[32 + j]) * sc;
+            }
+          }
         }
         tc_fence_before();
         asm volatile("bar.sync 1, 128;" ::: "memory");  // inv_l / l_part are reused by the next segment

@@ -78,3 +78,39 @@ def test_batch4_at_131072():
 def test_qwen_like_two_query_positions_batch64():
     seqlens = synth.uniform_seqlens(64, 2048, 8192, seed=5)
     check_sampled(synth.QWEN25_72B, seqlens, seed=5)
+
+
+# ------------------------------------------------------------------ every output at full size, by closed forms
+@pytest.mark.parametrize('shape,B', [(synth.LLAMA2_7B, 16), (synth.QWEN25_72B, 8)])
+def test_full_size_closed_forms_cover_every_output(shape, B):
+    """Two properties that hold at any size and fix every output element of a full-size launch:
+    identical cached rows give out = W_UV_h c whatever the queries are, and a zero softmax scale gives
+    out = W_UV_h mean_j(c_j) with lse = ln(visible tokens)."""
+    seqlens = [8192] * B
+    case = synth.make_decode_case(shape, seqlens, seed=23, device='cuda')
+    w_uv = lifts.f64(case['w_uv'])
+    # (1) zero scale on the random cache
+    out, lse, status, _, _ = gu.gpu_decode(shape, case, 0.0, G=0)
+    assert status == 0
+    got, got_lse = lifts.f64(out), lifts.f64(lse)
+    for b in range(B):
+        idx = case['page_table'][b, :8192 // 64].long()
+        rows = case['cache'][idx].reshape(-1, shape.row)[:, :shape.r].double()
+        for s in range(shape.S):
+            n = 8192 - (shape.S - 1 - s)
+            want = w_uv @ rows[:n].mean(0).cpu().numpy()                      # [H, dv]
+            gu.assert_close(got[b, s], want, f'uniform mean b={b} s={s}')
+            assert np.abs(got_lse[b, s] - np.log(n)).max() < 1e-3
+    # (2) every row of a sequence equal to its first row, ordinary scale
+    for b in range(B):
+        idx = case['page_table'][b, :8192 // 64].long()
+        first = case['cache'][idx[0], 0].clone()
+        case['cache'][idx] = first
+    out, _, status, _, _ = gu.gpu_decode(shape, case, gu.mla_scale(shape), G=0)
+    assert status == 0
+    got = lifts.f64(out)
+    for b in range(B):
+        c = lifts.f64(case['cache'][case['page_table'][b, 0].long(), 0, :shape.r])
+        want = w_uv @ c
+        for s in range(shape.S):
+            gu.assert_close(got[b, s], want, f'identical rows b={b} s={s}')
