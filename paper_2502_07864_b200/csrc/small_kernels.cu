@@ -226,17 +226,20 @@ __device__ void append_block(const __nv_bfloat16* __restrict__ x, const __nv_bfl
                              const int32_t* __restrict__ pos_base, int pos_shift,
                              const int32_t* __restrict__ page_table, __nv_bfloat16* __restrict__ cache,
                              int32_t* dev_status, int B, int S, int D, int r, int dR, int num_pages, int max_pages,
-                             float theta, int nb, unsigned char* smem_raw) {
+                             float theta, int nb, int t_splits, unsigned char* smem_raw) {
   float* red = reinterpret_cast<float*>(smem_raw);  // [8 warps][128 rows][8]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, t4 = lane & 3;
-  const int K = r + dR, f0 = nb * 8, T = B * S;
+  // block nb = (token split, feature tile): with many tokens the token range is cut so that more SMs take part
+  const int K = r + dR, f_tiles = K / 8, f0 = (nb % f_tiles) * 8;
+  const int t_chunk = (((B * S + t_splits - 1) / t_splits) + 15) & ~15;
+  const int t_begin = (nb / f_tiles) * t_chunk, T = min(B * S, t_begin + t_chunk);
   const int slice = D / 8, k_lo = warp * slice;
   const __nv_bfloat16* wrow = w + static_cast<size_t>(f0 + g) * D + k_lo + t4 * 8;
   if (t4 == 0)
     for (int k = 0; k < slice; k += 64) prefetch_l2(wrow + k);  // 128-byte lines of this warp's 8 weight rows
   pdl_wait();  // activations, positions and the cache may belong to kernels still in flight; the weights may not
-  for (int t0 = 0; t0 < T; t0 += kAppendMaxMT * 16) {
+  for (int t0 = t_begin; t0 < T; t0 += kAppendMaxMT * 16) {
     float acc[kAppendMaxMT][4];
 #pragma unroll
     for (int mt = 0; mt < kAppendMaxMT; ++mt) acc[mt][0] = acc[mt][1] = acc[mt][2] = acc[mt][3] = 0.f;
@@ -296,11 +299,11 @@ __global__ void __launch_bounds__(256) append_kernel(const __nv_bfloat16* __rest
                                                      const int32_t* __restrict__ page_table,
                                                      __nv_bfloat16* __restrict__ cache, int32_t* dev_status, int B,
                                                      int S, int D, int r, int dR, int num_pages, int max_pages,
-                                                     float theta) {
+                                                     float theta, int t_splits) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   pdl_trigger();
   append_block(x, w, positions, 0, page_table, cache, dev_status, B, S, D, r, dR, num_pages, max_pages, theta,
-               blockIdx.x, smem_raw);
+               blockIdx.x, t_splits, smem_raw);
 }
 
 // Absorb blocks followed by one plan block: everything transmla_mla_decode needs before the split-KV kernel.
@@ -329,18 +332,18 @@ __global__ void __launch_bounds__(256) prologue_kernel(
     const int32_t* __restrict__ page_table, __nv_bfloat16* __restrict__ cache, const __nv_bfloat16* __restrict__ q_nope,
     const __nv_bfloat16* __restrict__ q_pe, const __nv_bfloat16* __restrict__ w_uk, __nv_bfloat16* __restrict__ q_hat,
     const int32_t* __restrict__ seqlens, int32_t* cum, int32_t* plan, int32_t* dev_status, int B, int S, int H, int D,
-    int dn, int dR, int r, int num_pages, int max_pages, float theta, int G) {
+    int dn, int dR, int r, int num_pages, int max_pages, float theta, int G, int t_splits) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   pdl_trigger();
   TRK_BEGIN(0);
-  const int n_append = (r + dR) / 8;
+  const int n_append = (r + dR) / 8 * t_splits;
   const int r_tiles = (r + 127) / 128;
   const int bid = static_cast<int>(blockIdx.x) - 1;
   if (bid < 0) {
     plan_block(seqlens, B, G, cum, plan, smem_raw);
   } else if (bid < n_append) {
     append_block(x, w_dkv_kr, seqlens, -S, page_table, cache, dev_status, B, S, D, r, dR, num_pages, max_pages, theta,
-                 bid, smem_raw);
+                 bid, t_splits, smem_raw);
   } else {
     const int a = bid - n_append;
     absorb_block(q_nope, q_pe, w_uk, q_hat, B * S, H, dn, dR, r, a / r_tiles, a % r_tiles, smem_raw);
@@ -350,13 +353,20 @@ __global__ void __launch_bounds__(256) prologue_kernel(
 
 constexpr int kPrologueMaxSmem = 144 * 1024;
 
+// Token splits of the append: one per 64 new tokens, at most 4.
+static int append_token_splits(const transmla_params_t& p) {
+  const int T = p.batch * p.q_len;
+  return T <= 64 ? 1 : (T + 63) / 64 > 4 ? 4 : (T + 63) / 64;
+}
+
 cudaError_t launch_append(const transmla_params_t& p, const __nv_bfloat16* x, const __nv_bfloat16* w,
                           const int32_t* positions, const int32_t* page_table, __nv_bfloat16* cache,
                           int32_t* dev_status, cudaStream_t stream) {
   const int K = p.kv_lora_rank + p.qk_rope_dim;
-  return launch_pdl(append_kernel, dim3(K / 8), dim3(256), kAppendSmem, stream, x, w, positions, page_table, cache,
+  const int ts = append_token_splits(p);
+  return launch_pdl(append_kernel, dim3(K / 8 * ts), dim3(256), kAppendSmem, stream, x, w, positions, page_table, cache,
                     dev_status, p.batch, p.q_len, p.hidden_dim, p.kv_lora_rank, p.qk_rope_dim, p.num_pages,
-                    p.max_pages_per_seq, p.rope_theta);
+                    p.max_pages_per_seq, p.rope_theta, ts);
 }
 
 cudaError_t launch_absorb_plan(const transmla_params_t& p, int G, const __nv_bfloat16* q_nope,
@@ -388,10 +398,11 @@ cudaError_t launch_prologue(const transmla_params_t& p, int G, const __nv_bfloat
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  const int blocks = 1 + (p.kv_lora_rank + p.qk_rope_dim) / 8 + p.num_heads * ((p.kv_lora_rank + 127) / 128);
+  const int ts = append_token_splits(p);
+  const int blocks = 1 + (p.kv_lora_rank + p.qk_rope_dim) / 8 * ts + p.num_heads * ((p.kv_lora_rank + 127) / 128);
   return launch_pdl(prologue_kernel, dim3(blocks), dim3(256), smem, stream, x, w_dkv_kr, page_table, cache, q_nope, q_pe,
                     w_uk, q_hat, seqlens, cum, plan, dev_status, p.batch, p.q_len, p.num_heads, p.hidden_dim,
-                    p.qk_nope_dim, p.qk_rope_dim, p.kv_lora_rank, p.num_pages, p.max_pages_per_seq, p.rope_theta, G);
+                    p.qk_nope_dim, p.qk_rope_dim, p.kv_lora_rank, p.num_pages, p.max_pages_per_seq, p.rope_theta, G, ts);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -406,7 +417,10 @@ cudaError_t launch_prologue(const transmla_params_t& p, int G, const __nv_bfloat
 // ------------------------------------------------------------------------------------------------
 constexpr int kCombineRows = 16;
 
-__global__ void __launch_bounds__(256) combine_kernel(const int32_t* __restrict__ cum,
+// kPrefetch: hold the first weight tile in registers from before the dependency wait (few blocks, latency
+// matters); otherwise load weights window by window and keep the register count low enough for two blocks per SM.
+template <bool kPrefetch>
+__global__ void __launch_bounds__(256, kPrefetch ? 1 : 2) combine_kernel(const int32_t* __restrict__ cum,
                                                       const float* __restrict__ partial_o,
                                                       const float* __restrict__ partial_lse,
                                                       const __nv_bfloat16* __restrict__ w_uv,
@@ -426,9 +440,9 @@ __global__ void __launch_bounds__(256) combine_kernel(const int32_t* __restrict_
   const int nt_lo = blockIdx.z * tiles_per_z, nt_hi = min(tiles, nt_lo + tiles_per_z);
   // The weights do not depend on the merge: the first tile's 16-byte loads are issued now and land while
   // the partials are merged.
-  constexpr int kWin = 16;  // windows of 32 columns held in registers (r <= 512 fits one round)
+  constexpr int kWin = kPrefetch ? 16 : 4;  // windows of 32 columns held in registers per round
   uint4 wv[kWin];
-  {
+  if (kPrefetch) {
     const int nt = nt_lo + warp;
     const __nv_bfloat16* wrow = w_uv + (static_cast<size_t>(h) * dv + min(nt, tiles - 1) * 8 + g) * r + t4 * 8;
 #pragma unroll
@@ -527,7 +541,7 @@ __global__ void __launch_bounds__(256) combine_kernel(const int32_t* __restrict_
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
     const __nv_bfloat16* wrow = w_uv + (static_cast<size_t>(h) * dv + nt * 8 + g) * r + t4 * 8;
     for (int w0 = 0; w0 < r; w0 += kWin * 32) {  // kWin windows per round, all their loads in flight together
-      if (nt != nt_lo + warp || w0 != 0) {
+      if (!kPrefetch || nt != nt_lo + warp || w0 != 0) {
 #pragma unroll
         for (int u = 0; u < kWin; ++u)
           wv[u] = (w0 + u * 32 < r) ? ld_u128(wrow + w0 + u * 32) : make_uint4(0, 0, 0, 0);
@@ -567,7 +581,10 @@ cudaError_t launch_combine(const transmla_params_t& p, int G, const int32_t* cum
   const int zsplit = (BS <= 64 && p.v_dim >= 128) ? 2 : 1;
   dim3 grid(p.num_heads, (BS + rows - 1) / rows, zsplit);
   const size_t smem = 2 * kCombineRows * (p.kv_lora_rank + 8) * sizeof(__nv_bfloat16);
-  return launch_pdl(combine_kernel, grid, dim3(256), smem, stream, cum, partial_o, partial_lse, w_uv, out, lse_out,
+  if (BS <= 32)
+    return launch_pdl(combine_kernel<true>, grid, dim3(256), smem, stream, cum, partial_o, partial_lse, w_uv, out, lse_out,
+                      p.batch, p.q_len, p.num_heads, p.kv_lora_rank, p.v_dim, G, rows);
+  return launch_pdl(combine_kernel<false>, grid, dim3(256), smem, stream, cum, partial_o, partial_lse, w_uv, out, lse_out,
                     p.batch, p.q_len, p.num_heads, p.kv_lora_rank, p.v_dim, G, rows);
 }
 

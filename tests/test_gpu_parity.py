@@ -221,7 +221,9 @@ def test_a_wait_that_nothing_satisfies_ends_by_itself_and_leaves_the_context_usa
 
 # ------------------------------------------------------------------ append
 @pytest.mark.parametrize('shape,positions', [(synth.TINY, [16, 63, 64, 0]), (synth.LLAMA2_7B, [8191, 0, 77, 131071]),
-                                             (synth.QWEN25_72B, [126, 63, 4000])])
+                                             (synth.QWEN25_72B, [126, 63, 4000]),
+                                             (synth.TINY, [(7 * i) % 200 for i in range(150)]),       # several token splits
+                                             (synth.LLAMA2_7B, [(64 * i + i) % 700 for i in range(70)])])
 def test_append_values_slots_and_untouched_bytes(shape, positions):
     B, S, P = len(positions), shape.S, shape.page_size
     seqlens = [p + S for p in positions]
