@@ -289,3 +289,50 @@ def latent_append(x, w_dkv_kr, positions, page_table, cache, r, theta=10000.0, p
         page, off = append_slot(page_table[b], int(positions[b]), page_size)
         cache[page, off] = y
     return cache
+
+
+# --------------------------------------------------------------------------------------------
+# The steps either side of the attention: queries (Eq. 8, right column) and output projection
+# (Eq. 9, last line).  Used by the layer-level entry point.
+# --------------------------------------------------------------------------------------------
+def mla_queries(x, positions, w_uq, w_qr, H, w_dq=None, theta=10000.0):
+    """q^C and q^R of Eq. 8 (right column) for tokens x [T, D] at 0-based positions [T].
+
+    Low-rank queries: c^Q = W_DQ x, q^C = W_UQ c^Q, q^R = RoPE(W_QR c^Q, t).  With w_dq = None the
+    compression is skipped (full-rank queries: c^Q = x), which is the other variant the paper runs.
+    w_uq [H*dn, Dq], w_qr [H*dR, Dq].  Returns q_nope [T, H, dn] and q_pe [T, H, dR]; RoPE acts on each
+    head's dR-vector with d := dR.
+    """
+    x = np.asarray(x, np.float64)
+    c_q = x if w_dq is None else x @ np.asarray(w_dq, np.float64).T
+    T = x.shape[0]
+    q_nope = (c_q @ np.asarray(w_uq, np.float64).T).reshape(T, H, -1)
+    q_r = (c_q @ np.asarray(w_qr, np.float64).T).reshape(T, H, -1)
+    q_pe = rope(q_r, np.asarray(positions)[:, None], theta)
+    return q_nope, q_pe
+
+
+def output_projection(o, w_o):
+    """y_t = W_O [o_{t,1}; ...; o_{t,h}]  (Eq. 9, last line).  o [..., H, dv], w_o [D, H*dv]."""
+    o = np.asarray(o, np.float64)
+    return o.reshape(o.shape[:-2] + (-1,)) @ np.asarray(w_o, np.float64).T
+
+
+def mla_layer_decode(x, w_uq, w_qr, w_dkv_kr, w_uk, w_uv, w_o, cache, page_table, seqlens, scale, r,
+                     w_dq=None, theta=10000.0, page_size=64):
+    """One attention layer's decode step for the S newest tokens of every sequence, x [B, S, D] -> y [B, S, D].
+
+    Token (b, s) has position L_b - S + s.  Its latent row is appended (Eq. 7 left), queries are formed
+    (Eq. 8 right), attention runs in the MHA form over the cache (Eq. 8-9 left) and W_O is applied.  `cache` is
+    modified in place (float64).
+    """
+    x = np.asarray(x, np.float64)
+    B, S, _ = x.shape
+    H = w_uk.shape[0]
+    for s in range(S):
+        latent_append(x[:, s], w_dkv_kr, [int(L) - S + s for L in seqlens], page_table, cache, r, theta, page_size)
+    pos = np.array([[int(L) - S + s for s in range(S)] for L in seqlens])
+    q_nope, q_pe = mla_queries(x.reshape(B * S, -1), pos.reshape(-1), w_uq, w_qr, H, w_dq, theta)
+    o, _ = mla_decode_mha_form(q_nope.reshape(B, S, H, -1), q_pe.reshape(B, S, H, -1), w_uk, w_uv, cache, page_table,
+                               seqlens, scale, page_size)
+    return output_projection(o, w_o)

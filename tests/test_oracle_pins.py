@@ -383,6 +383,56 @@ def test_append_then_decode_equals_decode_over_the_full_sequence():
         assert np.allclose(out[0, 0, h], p @ (c @ w_uv[h].T), atol=1e-10)
 
 
+# ---------------------------------------------------------------- whole layer (Eq. 6 vs Eq. 10-14; App. A.2.2)
+def test_lifted_layer_reproduces_the_gqa_layer_output_token_by_token():
+    # A GQA layer decoded token by token through the MLA layer routine (cache built by its own appends) gives
+    # y_t = W_O [o_t,1; ...; o_t,h] of Eq. 6.  The lift keeps d^R = d rope dims for ALL key dims of one "rope
+    # head" per group is not available in the decoupled form, so the exact lift used here is g = 1 (MQA):
+    # W_KR = W_K (the single key head carries RoPE), the latent holds only the value head, W_UK is empty.
+    rng = np.random.default_rng(21)
+    h, d, D, T, P = 4, 8, 24, 9, 4
+    xs = rng.standard_normal((T, D))
+    w_q = rng.standard_normal((h * d, D)) / 5
+    w_k = rng.standard_normal((d, D)) / 5
+    w_v = rng.standard_normal((d, D)) / 5
+    w_o = rng.standard_normal((D, h * d)) / 5
+    # MLA weights: latent c = W_V x (r = d), rope key = RoPE(W_K x) (dR = d), no no-RoPE key part (dn = 0 is not
+    # representable, so one zero no-RoPE dim is carried: dn = 1 with zero W_UQ rows)
+    r, dR, dn = d, d, 1
+    w_dkv_kr = np.concatenate([w_v, w_k], axis=0)
+    w_uk = np.zeros((h, dn, r))
+    w_uv = np.tile(np.eye(d)[None], (h, 1, 1))
+    w_uq = np.zeros((h * dn, D))
+    table = np.array([[2, 0, 1]], dtype=np.int32)
+    cache = np.full((3, P, r + dR), np.nan)
+    for t in range(T):
+        y = orc.mla_layer_decode(xs[t][None, None], w_uq, w_q, w_dkv_kr, w_uk, w_uv, w_o, cache, table, [t + 1],
+                                 1.0 / np.sqrt(d), r, page_size=P)
+        ref = orc.gqa_attention_last_token(xs[:t + 1], w_q, w_k, w_v, h, 1)
+        assert np.abs(y[0, 0] - ref.reshape(-1) @ w_o.T).max() < 1e-10
+
+
+def test_low_rank_queries_and_folded_output_projection():
+    # Eq. 8 right: low-rank queries equal full-rank ones with W = W_U{Q,R} W_DQ; App. A.2.2: folding the block
+    # diagonal of W_UV into W_O gives the same y from the latent-space outputs.
+    rng = np.random.default_rng(22)
+    H, dn, dR, dv, r, D, rq, T = 3, 4, 6, 5, 7, 16, 8, 5
+    x = rng.standard_normal((T, D))
+    w_dq, w_uq, w_qr = rng.standard_normal((rq, D)), rng.standard_normal((H * dn, rq)), rng.standard_normal((H * dR, rq))
+    pos = np.array([0, 3, 3, 100, 7])
+    a = orc.mla_queries(x, pos, w_uq, w_qr, H, w_dq)
+    b = orc.mla_queries(x, pos, w_uq @ w_dq, w_qr @ w_dq, H)
+    assert np.abs(a[0] - b[0]).max() < 1e-9 and np.abs(a[1] - b[1]).max() < 1e-9
+    # RoPE really sits on the rope part, per head, at the token's position
+    raw = (x @ (w_qr @ w_dq).T).reshape(T, H, dR)
+    assert np.abs(a[1][3, 1] - orc.rope(raw[3, 1], 100)).max() < 1e-9 and np.abs(a[1][0] - raw[0]).max() < 1e-12
+    o_lat = rng.standard_normal((T, H, r))
+    w_uv, w_o = rng.standard_normal((H, dv, r)), rng.standard_normal((D, H * dv))
+    o = np.einsum('hvr,thr->thv', w_uv, o_lat)
+    folded = np.concatenate([w_o[:, i * dv:(i + 1) * dv] @ w_uv[i] for i in range(H)], axis=1)      # W'O [D, H*r]
+    assert np.abs(orc.output_projection(o, w_o) - o_lat.reshape(T, -1) @ folded.T).max() < 1e-9
+
+
 # ---------------------------------------------------------------- numbers the paper prints
 def test_kv_cache_ratio_printed_in_the_paper():
     here = os.path.dirname(os.path.abspath(__file__))
