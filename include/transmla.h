@@ -176,6 +176,36 @@ transmla_status_t transmla_decode_step(const transmla_params_t* params /* host *
                                        size_t workspace_bytes, void* out, float* lse_out, int32_t* dev_status,
                                        void* stream);
 
+/* Weights of one converted attention layer for transmla_layer_decode_step (all device bf16, row-major).
+ * Queries follow Eq. 8, right column: c^Q = W_DQ x, q^C = W_UQ c^Q, q^R = RoPE(W_QR c^Q, t).  With
+ * w_dq == NULL the compression is skipped (full-rank queries, the other variant the paper runs): w_uq and
+ * w_qr then act on x itself. */
+typedef struct {
+  const void* w_dq;      /* [r_q, D] or NULL */
+  int32_t q_lora_rank;   /* r_q (multiple of 256); ignored when w_dq == NULL */
+  const void* w_uq;      /* [H*dn, Dq], Dq = r_q or D: rows h*dn .. h*dn+dn-1 give q^C of head h */
+  const void* w_qr;      /* [H*dR, Dq]: rows h*dR .. give q^R of head h before RoPE (NULL when dR == 0) */
+  const void* w_dkv_kr;  /* [r+dR, D]   as in transmla_latent_append */
+  const void* w_uk;      /* [H, dn, r]  as in transmla_mla_decode */
+  const void* w_uv;      /* [H, dv, r]  as in transmla_mla_combine */
+  const void* w_o;       /* [D, H*dv]:  y = W_O [o_1; ...; o_H]  (Eq. 9, last line) */
+} transmla_layer_weights_t;
+
+/* Bytes of device scratch transmla_layer_decode_step needs (c^Q, q^C, q^R and the attention output, bf16). */
+size_t transmla_layer_scratch_bytes(const transmla_params_t* params /* host */, int32_t q_lora_rank);
+
+/* The whole attention layer for the S newest tokens of every sequence, x [B, S, D] -> y [B, S, D] (device bf16):
+ * queries (Eq. 8 right column, RoPE of q^R at position L_b - S + s), then transmla_decode_step (append, absorb,
+ * split-KV decode, combine), then the output projection W_O (Eq. 9, last line).  The linear maps are skinny
+ * GEMMs with M = B*S that stream their weights once.  Needs D, H*dv (and r_q) multiples of 256; other rules
+ * as for transmla_decode_step.  `scratch` is device memory of transmla_layer_scratch_bytes bytes, 256-byte
+ * aligned. */
+transmla_status_t transmla_layer_decode_step(const transmla_params_t* params /* host */,
+                                             const transmla_layer_weights_t* weights /* host struct of device ptrs */,
+                                             const void* x, const int32_t* page_table, const int32_t* seqlens,
+                                             void* cache, void* workspace, size_t workspace_bytes, void* scratch,
+                                             size_t scratch_bytes, void* y, int32_t* dev_status, void* stream);
+
 /* Bytes of device staging transmla_decode_step_host needs for `params`. */
 size_t transmla_step_staging_bytes(const transmla_params_t* params /* host */);
 

@@ -14,7 +14,8 @@ _LIB_PATH = os.path.join(_HERE, 'libtransmla.so')
 EXPORTS = ('transmla_workspace_layout', 'transmla_latent_append', 'transmla_mla_decode', 'transmla_mla_combine',
            'transmla_validate_tables', 'transmla_step_staging_bytes', 'transmla_decode_step_host',
            'transmla_decode_step', 'transmla_profile_decode_kernel', 'transmla_status_string',
-           'transmla_static_workspace_capacity', 'transmla_mla_attention_static', 'transmla_selftest_bounded_wait')
+           'transmla_static_workspace_capacity', 'transmla_mla_attention_static', 'transmla_selftest_bounded_wait',
+           'transmla_layer_scratch_bytes', 'transmla_layer_decode_step')
 
 
 class Params(ctypes.Structure):
@@ -29,6 +30,12 @@ class WorkspaceLayout(ctypes.Structure):
                 ('q_hat_offset', ctypes.c_size_t), ('cum_pages_offset', ctypes.c_size_t),
                 ('plan_offset', ctypes.c_size_t), ('partial_o_offset', ctypes.c_size_t),
                 ('partial_lse_offset', ctypes.c_size_t), ('total_bytes', ctypes.c_size_t)]
+
+
+class LayerWeights(ctypes.Structure):
+    _fields_ = [('w_dq', ctypes.c_void_p), ('q_lora_rank', ctypes.c_int32), ('w_uq', ctypes.c_void_p),
+                ('w_qr', ctypes.c_void_p), ('w_dkv_kr', ctypes.c_void_p), ('w_uk', ctypes.c_void_p),
+                ('w_uv', ctypes.c_void_p), ('w_o', ctypes.c_void_p)]
 
 
 class TransMLAError(RuntimeError):
@@ -65,11 +72,16 @@ def lib():
         L.transmla_static_workspace_capacity.restype = sz
         L.transmla_mla_attention_static.argtypes = [pp, vp, vp, vp, vp, vp, i32p, i32p, vp, vp, i32p, vp]
         L.transmla_selftest_bounded_wait.argtypes = [i32p, vp, vp]
+        L.transmla_layer_scratch_bytes.argtypes = [pp, ctypes.c_int32]
+        L.transmla_layer_scratch_bytes.restype = sz
+        L.transmla_layer_decode_step.argtypes = [pp, ctypes.POINTER(LayerWeights), vp, i32p, i32p, vp, vp, sz, vp, sz, vp,
+                                                 i32p, vp]
         L.transmla_status_string.argtypes = [ctypes.c_int]
         L.transmla_status_string.restype = ctypes.c_char_p
         for name in EXPORTS:
             if name not in ('transmla_step_staging_bytes', 'transmla_status_string',
-                            'transmla_profile_decode_kernel', 'transmla_static_workspace_capacity'):
+                            'transmla_profile_decode_kernel', 'transmla_static_workspace_capacity',
+                            'transmla_layer_scratch_bytes'):
                 getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -170,6 +182,24 @@ def transmla_mla_attention_static(params, q_nope, q_pe, w_uk, w_uv, cache, page_
     _check(lib().transmla_mla_attention_static(
         ctypes.byref(params), _ptr(q_nope), _ptr(q_pe), _ptr(w_uk), _ptr(w_uv), _ptr(cache), _ptr(page_table),
         _ptr(seqlens), _ptr(out), _ptr(lse_out), _ptr(dev_status), _stream(stream)), 'transmla_mla_attention_static')
+
+
+def transmla_layer_scratch_bytes(params, q_lora_rank=0):
+    return lib().transmla_layer_scratch_bytes(ctypes.byref(params), int(q_lora_rank))
+
+
+def transmla_layer_decode_step(params, weights, x, page_table, seqlens, cache, workspace, scratch, y, dev_status=None,
+                               stream=None):
+    """weights: dict of device tensors w_uq, w_qr, w_dkv_kr, w_uk, w_uv, w_o and optionally w_dq (low-rank queries)."""
+    w_dq = weights.get('w_dq')
+    lw = LayerWeights(w_dq=None if w_dq is None else w_dq.data_ptr(), q_lora_rank=0 if w_dq is None else w_dq.shape[0],
+                      w_uq=weights['w_uq'].data_ptr(), w_qr=None if weights.get('w_qr') is None else weights['w_qr'].data_ptr(),
+                      w_dkv_kr=weights['w_dkv_kr'].data_ptr(), w_uk=weights['w_uk'].data_ptr(),
+                      w_uv=weights['w_uv'].data_ptr(), w_o=weights['w_o'].data_ptr())
+    _check(lib().transmla_layer_decode_step(
+        ctypes.byref(params), ctypes.byref(lw), _ptr(x), _ptr(page_table), _ptr(seqlens), _ptr(cache), _ptr(workspace),
+        workspace.numel() * workspace.element_size(), _ptr(scratch), scratch.numel() * scratch.element_size(), _ptr(y),
+        _ptr(dev_status), _stream(stream)), 'transmla_layer_decode_step')
 
 
 def transmla_selftest_bounded_wait(dev_status, cycles_out=None, stream=None):

@@ -1,0 +1,125 @@
+// Linear maps either side of the attention (Eq. 8 right column: queries; Eq. 9 last line: W_O), as skinny GEMMs
+// y[M, N] = x[M, K] w[N, K]^T with M = the step's new tokens.  They stream their weights once; a block owns 8
+// output features (see skinny_gemm.cuh).  One launch may hold two jobs (q^C and q^R share their input).
+#include "common.cuh"
+#include "skinny_gemm.cuh"
+
+namespace transmla {
+
+struct LinearJob {
+  const __nv_bfloat16* x;   // [M, K]
+  const __nv_bfloat16* w;   // [N, K]
+  __nv_bfloat16* out;       // [M, N]
+  int N, K;
+  int rope_d;               // > 0: consecutive blocks of rope_d output features are rotated (Eq. 1, d := rope_d)
+};
+struct LinearArgs {
+  LinearJob job[2];
+  int n_jobs, M, S, t_splits;
+  const int32_t* pos_base;  // position of token (b, s) = pos_base[b] + pos_shift + s (used by rotated jobs only)
+  int pos_shift;
+  float theta;
+};
+
+__global__ void __launch_bounds__(256) linear_kernel(LinearArgs a) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  pdl_trigger();
+  int nb = blockIdx.x, j = 0;
+  const int blocks0 = a.job[0].N / 8 * a.t_splits;
+  if (a.n_jobs > 1 && nb >= blocks0) { nb -= blocks0; j = 1; }
+  const LinearJob job = a.job[j];
+  const int f_tiles = job.N / 8, f0 = (nb % f_tiles) * 8;
+  const int t_chunk = (((a.M + a.t_splits - 1) / a.t_splits) + 15) & ~15;
+  const int t_begin = (nb / f_tiles) * t_chunk, t_end = min(a.M, t_begin + t_chunk);
+  skinny_gemm_tile(job.x, job.w, job.K, f0, t_begin, t_end, smem_raw, [&](int t, int pr, float re, float im) {
+    const int f = f0 + pr * 2;
+    if (job.rope_d > 0) {
+      const int pos = a.pos_base[t / a.S] + a.pos_shift + t % a.S;
+      rope_pair(re, im, pos, (f % job.rope_d) >> 1, job.rope_d, a.theta);
+    }
+    *reinterpret_cast<uint32_t*>(job.out + static_cast<size_t>(t) * job.N + f) = pack_bf16(re, im);
+  });
+}
+
+cudaError_t launch_linear(const LinearArgs& args, cudaStream_t stream) {
+  int blocks = 0;
+  for (int j = 0; j < args.n_jobs; ++j) blocks += args.job[j].N / 8 * args.t_splits;
+  return launch_pdl(linear_kernel, dim3(blocks), dim3(256), kAppendSmem, stream, args);
+}
+
+}  // namespace transmla
+
+using namespace transmla;
+
+namespace {
+constexpr size_t kAlign = 256;
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+inline int token_splits(int M) { return M <= 64 ? 1 : (M + 63) / 64 > 4 ? 4 : (M + 63) / 64; }
+}  // namespace
+
+extern "C" {
+
+size_t transmla_layer_scratch_bytes(const transmla_params_t* p, int32_t q_lora_rank) {
+  if (p == nullptr || q_lora_rank < 0) return 0;
+  const size_t M = static_cast<size_t>(p->batch) * p->q_len, H = p->num_heads;
+  size_t off = 0;
+  off = round_up(off + M * q_lora_rank * 2, kAlign);
+  off = round_up(off + M * H * p->qk_nope_dim * 2, kAlign);
+  off = round_up(off + M * H * p->qk_rope_dim * 2 + 16, kAlign);
+  off = round_up(off + M * H * p->v_dim * 2, kAlign);
+  return off;
+}
+
+transmla_status_t transmla_layer_decode_step(const transmla_params_t* p, const transmla_layer_weights_t* w,
+                                             const void* x, const int32_t* page_table, const int32_t* seqlens,
+                                             void* cache, void* workspace, size_t workspace_bytes, void* scratch,
+                                             size_t scratch_bytes, void* y, int32_t* dev_status, void* stream) {
+  if (p == nullptr || w == nullptr) return TRANSMLA_ERR_NULL;
+  if (!x || !seqlens || !scratch || !y || !w->w_uq || !w->w_o || !w->w_dkv_kr || !w->w_uk || !w->w_uv) return TRANSMLA_ERR_NULL;
+  if (p->qk_rope_dim > 0 && !w->w_qr) return TRANSMLA_ERR_NULL;
+  const bool low_rank = w->w_dq != nullptr;
+  const int H = p->num_heads, D = p->hidden_dim, rq = low_rank ? w->q_lora_rank : 0;
+  const int Kq = low_rank ? rq : D, Ko = H * p->v_dim;
+  if (p->batch < 1 || p->q_len < 1 || D < 256 || D % 256 || Ko % 256 || (low_rank && (rq < 256 || rq % 256)) ||
+      (H * p->qk_nope_dim) % 8 || (H * p->qk_rope_dim) % 8 || p->qk_rope_dim % 2)
+    return TRANSMLA_ERR_SHAPE;
+  if (!aligned16(x) || !aligned16(y) || !aligned16(w->w_dq) || !aligned16(w->w_uq) || !aligned16(w->w_qr) ||
+      !aligned16(w->w_o) || (reinterpret_cast<uintptr_t>(scratch) & (kAlign - 1)))
+    return TRANSMLA_ERR_ALIGN;
+  if (scratch_bytes < transmla_layer_scratch_bytes(p, rq)) return TRANSMLA_ERR_WORKSPACE;
+
+  const int M = p->batch * p->q_len;
+  char* base = static_cast<char*>(scratch);
+  size_t off = 0;
+  auto* cq = reinterpret_cast<__nv_bfloat16*>(base + off);      off = round_up(off + static_cast<size_t>(M) * rq * 2, kAlign);
+  auto* q_nope = reinterpret_cast<__nv_bfloat16*>(base + off);  off = round_up(off + static_cast<size_t>(M) * H * p->qk_nope_dim * 2, kAlign);
+  auto* q_pe = reinterpret_cast<__nv_bfloat16*>(base + off);    off = round_up(off + static_cast<size_t>(M) * H * p->qk_rope_dim * 2 + 16, kAlign);
+  auto* attn = reinterpret_cast<__nv_bfloat16*>(base + off);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const auto* xin = static_cast<const __nv_bfloat16*>(x);
+
+  LinearArgs a = {};
+  a.M = M; a.S = p->q_len; a.t_splits = token_splits(M); a.pos_base = seqlens; a.pos_shift = -p->q_len; a.theta = p->rope_theta;
+  if (low_rank) {  // c^Q = W_DQ x
+    a.n_jobs = 1;
+    a.job[0] = {xin, static_cast<const __nv_bfloat16*>(w->w_dq), cq, rq, D, 0};
+    if (launch_linear(a, s) != cudaSuccess) return TRANSMLA_ERR_CUDA;
+  }
+  const __nv_bfloat16* qin = low_rank ? cq : xin;
+  a.n_jobs = p->qk_rope_dim > 0 ? 2 : 1;  // q^C = W_UQ c^Q and q^R = RoPE(W_QR c^Q, t) in one launch
+  a.job[0] = {qin, static_cast<const __nv_bfloat16*>(w->w_uq), q_nope, H * p->qk_nope_dim, Kq, 0};
+  a.job[1] = {qin, static_cast<const __nv_bfloat16*>(w->w_qr), q_pe, H * p->qk_rope_dim, Kq, p->qk_rope_dim};
+  if (launch_linear(a, s) != cudaSuccess) return TRANSMLA_ERR_CUDA;
+
+  transmla_status_t st = transmla_decode_step(p, x, q_nope, q_pe, page_table, seqlens, w->w_dkv_kr, w->w_uk, w->w_uv, cache,
+                                              workspace, workspace_bytes, attn, nullptr, dev_status, stream);
+  if (st != TRANSMLA_OK) return st;
+
+  a.n_jobs = 1;  // y = W_O [o_1; ...; o_h]
+  a.job[0] = {attn, static_cast<const __nv_bfloat16*>(w->w_o), static_cast<__nv_bfloat16*>(y), D, Ko, 0};
+  if (launch_linear(a, s) != cudaSuccess) return TRANSMLA_ERR_CUDA;
+  return TRANSMLA_OK;
+}
+
+}  // extern "C"

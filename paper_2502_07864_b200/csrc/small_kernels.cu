@@ -12,6 +12,7 @@
 // (x, y) to one MMA and (z, w) to the next.  Where one operand comes from shared memory instead, it
 // is stored there in the matching order (kperm below).
 #include "common.cuh"
+#include "skinny_gemm.cuh"
 
 namespace transmla {
 
@@ -35,8 +36,6 @@ extern "C" int transmla_ktrace_dump(unsigned long long* host, int reset) {
 #define TRCK(ev) do { } while (0)
 #endif
 
-__device__ __forceinline__ uint32_t ld_u32(const __nv_bfloat16* p) { return *reinterpret_cast<const uint32_t*>(p); }
-__device__ __forceinline__ uint4 ld_u128(const __nv_bfloat16* p) { return *reinterpret_cast<const uint4*>(p); }
 
 // Position, inside its 32-wide window, at which element p must sit in shared memory so that ldmatrix
 // hands out the fragment that pairs with a uint4 global load of the other operand.
@@ -189,108 +188,29 @@ static size_t absorb_smem(int dn) {
 // split the hidden dimension and meet in shared memory.  Tokens are the M dimension of the tiles.
 // Token (b, s) sits at position pos_base[b] + pos_shift + s.
 // ------------------------------------------------------------------------------------------------
-constexpr int kAppendMaxMT = 8;  // 16-token tiles per pass
-constexpr size_t kAppendSmem = 8 * kAppendMaxMT * 16 * 8 * sizeof(float);  // 32 KB
-
-// Partial products of one warp over its slice of the hidden dimension for tokens [t0, t0 + 16*MT).
-template <int MT, int UNROLL>
-__device__ __forceinline__ void append_partial(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ wrow,
-                                               int D, int T, int t0, int k_lo, int slice, int g, int t4,
-                                               float (&acc)[kAppendMaxMT][4]) {
-  const __nv_bfloat16* xr[MT][2];
-  bool ok[MT][2];
-#pragma unroll
-  for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-    for (int hf = 0; hf < 2; ++hf) {
-      const int row = t0 + mt * 16 + g + hf * 8;
-      ok[mt][hf] = row < T;
-      xr[mt][hf] = x + static_cast<size_t>(min(row, T - 1)) * D + k_lo + t4 * 8;
-    }
-#pragma unroll UNROLL
-  for (int k = 0; k < slice; k += 32) {
-    const uint4 wv = ld_u128(wrow + k);
-#pragma unroll
-    for (int mt = 0; mt < MT; ++mt) {
-      uint4 x0 = make_uint4(0, 0, 0, 0), x1 = make_uint4(0, 0, 0, 0);
-      if (ok[mt][0]) x0 = ld_u128(xr[mt][0] + k);
-      if (ok[mt][1]) x1 = ld_u128(xr[mt][1] + k);
-      const uint32_t a0[4] = {x0.x, x1.x, x0.y, x1.y}, a1[4] = {x0.z, x1.z, x0.w, x1.w};
-      mma_bf16_16816(acc[mt], a0, wv.x, wv.y);
-      mma_bf16_16816(acc[mt], a1, wv.z, wv.w);
-    }
-  }
-}
-
 __device__ void append_block(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w,
                              const int32_t* __restrict__ pos_base, int pos_shift,
                              const int32_t* __restrict__ page_table, __nv_bfloat16* __restrict__ cache,
                              int32_t* dev_status, int B, int S, int D, int r, int dR, int num_pages, int max_pages,
                              float theta, int nb, int t_splits, unsigned char* smem_raw) {
-  float* red = reinterpret_cast<float*>(smem_raw);  // [8 warps][128 rows][8]
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int g = lane >> 2, t4 = lane & 3;
   // block nb = (token split, feature tile): with many tokens the token range is cut so that more SMs take part
   const int K = r + dR, f_tiles = K / 8, f0 = (nb % f_tiles) * 8;
   const int t_chunk = (((B * S + t_splits - 1) / t_splits) + 15) & ~15;
-  const int t_begin = (nb / f_tiles) * t_chunk, T = min(B * S, t_begin + t_chunk);
-  const int slice = D / 8, k_lo = warp * slice;
-  const __nv_bfloat16* wrow = w + static_cast<size_t>(f0 + g) * D + k_lo + t4 * 8;
-  if (t4 == 0)
-    for (int k = 0; k < slice; k += 64) prefetch_l2(wrow + k);  // 128-byte lines of this warp's 8 weight rows
-  pdl_wait();  // activations, positions and the cache may belong to kernels still in flight; the weights may not
-  for (int t0 = t_begin; t0 < T; t0 += kAppendMaxMT * 16) {
-    float acc[kAppendMaxMT][4];
-#pragma unroll
-    for (int mt = 0; mt < kAppendMaxMT; ++mt) acc[mt][0] = acc[mt][1] = acc[mt][2] = acc[mt][3] = 0.f;
-    const int left = T - t0;
-    if (left <= 16) append_partial<1, 8>(x, wrow, D, T, t0, k_lo, slice, g, t4, acc);
-    else if (left <= 32) append_partial<2, 4>(x, wrow, D, T, t0, k_lo, slice, g, t4, acc);
-    else if (left <= 64) append_partial<4, 4>(x, wrow, D, T, t0, k_lo, slice, g, t4, acc);
-    else append_partial<8, 2>(x, wrow, D, T, t0, k_lo, slice, g, t4, acc);
-    __syncthreads();  // previous pass has consumed `red`
-#pragma unroll
-    for (int mt = 0; mt < kAppendMaxMT; ++mt) {
-      if (mt * 16 < left) {
-        float* d = red + (warp * kAppendMaxMT * 16 + mt * 16 + g) * 8 + t4 * 2;
-        *reinterpret_cast<float2*>(d) = make_float2(acc[mt][0], acc[mt][1]);
-        *reinterpret_cast<float2*>(d + 64) = make_float2(acc[mt][2], acc[mt][3]);
-      }
+  const int t_begin = (nb / f_tiles) * t_chunk, t_end = min(B * S, t_begin + t_chunk);
+  skinny_gemm_tile(x, w, D, f0, t_begin, t_end, smem_raw, [&](int t, int pr, float re, float im) {
+    const int b = t / S, s = t % S;
+    const int pos = pos_base[b] + pos_shift + s;
+    const int pj = pos / kPage;
+    int page = -1;
+    if (pos >= 0 && pj < max_pages) page = page_table[static_cast<size_t>(b) * max_pages + pj];
+    if (page < 0 || page >= num_pages) {
+      set_status(dev_status, TRANSMLA_DEV_BAD_PAGE);
+      return;
     }
-    __syncthreads();
-    const int rows = min(kAppendMaxMT * 16, left);
-    for (int i = tid; i < rows * 4; i += 256) {
-      const int row = i >> 2, pr = i & 3;
-      float re = 0.f, im = 0.f;
-#pragma unroll
-      for (int wv = 0; wv < 8; ++wv) {
-        const float2 v = *reinterpret_cast<const float2*>(red + (wv * kAppendMaxMT * 16 + row) * 8 + pr * 2);
-        re += v.x; im += v.y;
-      }
-      const int t = t0 + row, b = t / S, s = t % S;
-      const int pos = pos_base[b] + pos_shift + s;
-      const int pj = pos / kPage;
-      int page = -1;
-      if (pos >= 0 && pj < max_pages) page = page_table[static_cast<size_t>(b) * max_pages + pj];
-      if (page < 0 || page >= num_pages) {
-        set_status(dev_status, TRANSMLA_DEV_BAD_PAGE);
-        continue;
-      }
-      const int f = f0 + pr * 2;
-      if (f >= r) {
-        // RoPE pair l (Eq. 1).  The angle is formed and reduced to [-pi, pi] in fp64 so that positions of
-        // 10^5 keep their phase; the sine and cosine of the reduced angle are fp32.
-        const int l = (f - r) >> 1;
-        const double ang = static_cast<double>(pos) * exp2(-2.0 * l / dR * log2(static_cast<double>(theta)));
-        const double red_ang = ang - 6.283185307179586476925 * rint(ang * 0.15915494309189533577);
-        float sn, cs;
-        sincosf(static_cast<float>(red_ang), &sn, &cs);
-        const float nre = re * cs - im * sn, nim = im * cs + re * sn;
-        re = nre; im = nim;
-      }
-      *reinterpret_cast<uint32_t*>(cache + (static_cast<size_t>(page) * kPage + pos % kPage) * K + f) = pack_bf16(re, im);
-    }
-  }
+    const int f = f0 + pr * 2;
+    if (f >= r) rope_pair(re, im, pos, (f - r) >> 1, dR, theta);  // RoPE pair l of the decoupled key (Eq. 1)
+    *reinterpret_cast<uint32_t*>(cache + (static_cast<size_t>(page) * kPage + pos % kPage) * K + f) = pack_bf16(re, im);
+  });
 }
 
 __global__ void __launch_bounds__(256) append_kernel(const __nv_bfloat16* __restrict__ x,

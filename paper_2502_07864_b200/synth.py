@@ -112,3 +112,18 @@ def make_append_case(shape, positions, seed, device='cpu'):
         'w_dkv_kr': _randn_bf16((shape.row, shape.D), shape.D ** -0.5, g, device),
         'positions': torch.tensor([int(p) for p in positions], dtype=torch.int32, device=device),
     }
+
+
+def make_layer_weights(shape, seed, q_lora_rank=0, device='cpu'):
+    """Weights of the linear maps either side of the attention: w_uq [H*dn, Dq], w_qr [H*dR, Dq], w_o [D, H*dv] and,
+    for low-rank queries, w_dq [r_q, D]; N(0, 1/sqrt(fan_in)), bf16."""
+    g = _gen(seed, device)
+    Dq = q_lora_rank if q_lora_rank else shape.D
+    w = {
+        'w_uq': _randn_bf16((shape.H * shape.dn, Dq), Dq ** -0.5, g, device),
+        'w_qr': _randn_bf16((shape.H * shape.dR, Dq), Dq ** -0.5, g, device),
+        'w_o': _randn_bf16((shape.D, shape.H * shape.dv), (shape.H * shape.dv) ** -0.5, g, device),
+    }
+    if q_lora_rank:
+        w['w_dq'] = _randn_bf16((q_lora_rank, shape.D), shape.D ** -0.5, g, device)
+    return w

@@ -284,3 +284,32 @@ def test_decode_step_from_host_buffers(pinned):
     want, want_lse = gu.oracle_decode(shape, case, scale)
     gu.assert_close(lifts.f64(h_out), want, 'host step')
     gu.assert_lse_close(lifts.f64(h_lse), want_lse, 'host step lse')
+
+
+# ------------------------------------------------------------------ whole layer: queries, attention, W_O
+@pytest.mark.parametrize('shape,seqlens,rq', [(synth.TINY, [17, 64, 130], 0), (synth.TINY, [5, 70], 256),
+                                               (synth.LLAMA2_7B, [300, 65, 1024], 0), (synth.LLAMA2_7B, [200, 64], 512),
+                                               (synth.QWEN25_72B, [131, 700], 0)])
+def test_layer_decode_step(shape, seqlens, rq):
+    B, S = len(seqlens), shape.S
+    scale = gu.mla_scale(shape)
+    dc = synth.make_decode_case(shape, seqlens, 31)
+    ac = synth.make_append_case(shape, [L - S for L in seqlens], 32)
+    lw = synth.make_layer_weights(shape, 33, q_lora_rank=rq)
+    weights = {k: v.cuda() for k, v in lw.items()}
+    weights.update(w_dkv_kr=ac['w_dkv_kr'].cuda(), w_uk=dc['w_uk'].cuda(), w_uv=dc['w_uv'].cuda())
+    params = binding.make_params(shape, B, dc['cache'].shape[0], dc['page_table'].shape[1], scale)
+    ws, _ = binding.alloc_workspace(params)
+    scratch = torch.empty(binding.transmla_layer_scratch_bytes(params, rq), dtype=torch.uint8, device='cuda')
+    y = torch.full((B, S, shape.D), float('nan'), dtype=torch.bfloat16, device='cuda')
+    status = torch.zeros(1, dtype=torch.int32, device='cuda')
+    cache = dc['cache'].cuda()
+    binding.transmla_layer_decode_step(params, weights, ac['x'].cuda(), dc['page_table'].cuda(), dc['seqlens'].cuda(), cache,
+                                       ws, scratch, y, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    want = orc.mla_layer_decode(lifts.f64(ac['x']), lifts.f64(lw['w_uq']), lifts.f64(lw['w_qr']), lifts.f64(ac['w_dkv_kr']),
+                                lifts.f64(dc['w_uk']), lifts.f64(dc['w_uv']), lifts.f64(lw['w_o']), lifts.f64(dc['cache']),
+                                dc['page_table'].numpy(), seqlens, scale, shape.r,
+                                w_dq=None if not rq else lifts.f64(lw['w_dq']))
+    err, rel = gu.assert_close(lifts.f64(y), want, f'layer output rq={rq}')
