@@ -21,17 +21,19 @@ struct LinearArgs {
   float theta;
 };
 
-__global__ void __launch_bounds__(256) linear_kernel(LinearArgs a) {
+// MAXMT x 16 tokens per pass, NT x 8 output features per block.
+template <int MAXMT, int NT>
+__global__ void __launch_bounds__(256, 1) linear_kernel(LinearArgs a) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   pdl_trigger();
   int nb = blockIdx.x, j = 0;
-  const int blocks0 = a.job[0].N / 8 * a.t_splits;
+  const int blocks0 = a.job[0].N / (8 * NT) * a.t_splits;
   if (a.n_jobs > 1 && nb >= blocks0) { nb -= blocks0; j = 1; }
   const LinearJob job = a.job[j];
-  const int f_tiles = job.N / 8, f0 = (nb % f_tiles) * 8;
+  const int f_tiles = job.N / (8 * NT), f0 = (nb % f_tiles) * 8 * NT;
   const int t_chunk = (((a.M + a.t_splits - 1) / a.t_splits) + 15) & ~15;
   const int t_begin = (nb / f_tiles) * t_chunk, t_end = min(a.M, t_begin + t_chunk);
-  skinny_gemm_tile(job.x, job.w, job.K, f0, t_begin, t_end, smem_raw, [&](int t, int pr, float re, float im) {
+  skinny_gemm_tile<MAXMT, NT>(job.x, job.w, job.K, f0, t_begin, t_end, smem_raw, [&](int t, int pr, float re, float im) {
     const int f = f0 + pr * 2;
     if (job.rope_d > 0) {
       const int pos = a.pos_base[t / a.S] + a.pos_shift + t % a.S;
@@ -42,9 +44,21 @@ __global__ void __launch_bounds__(256) linear_kernel(LinearArgs a) {
 }
 
 cudaError_t launch_linear(const LinearArgs& args, cudaStream_t stream) {
+  // 32 features per block when every job allows it (the activations are then read a quarter as often)
+  bool wide = true;
+  for (int j = 0; j < args.n_jobs; ++j) wide = wide && args.job[j].N % 32 == 0;
+  const int per_block = wide ? 32 : 8;
   int blocks = 0;
-  for (int j = 0; j < args.n_jobs; ++j) blocks += args.job[j].N / 8 * args.t_splits;
-  return launch_pdl(linear_kernel, dim3(blocks), dim3(256), kAppendSmem, stream, args);
+  for (int j = 0; j < args.n_jobs; ++j) blocks += args.job[j].N / per_block * args.t_splits;
+  if (!wide) return launch_pdl(linear_kernel<8, 1>, dim3(blocks), dim3(256), skinny_gemm_smem(8, 1), stream, args);
+  constexpr size_t smem = skinny_gemm_smem(4, 4);  // 64 KB: above the default limit
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(linear_kernel<4, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  return launch_pdl(linear_kernel<4, 4>, dim3(blocks), dim3(256), smem, stream, args);
 }
 
 }  // namespace transmla
