@@ -31,12 +31,14 @@ namespace sm100 {
 // Optional timeline instrumentation (compile with -DTRANSMLA_TRACE): clock64 stamps of one CTA's pipeline
 // events and the global-timer start/end of every CTA, read back with transmla_trace_dump().
 #ifdef TRANSMLA_TRACE
-__device__ long long g_trace[16][256];
+__device__ long long g_trace[24][256];
 #define TR(ev, idx) do { if (blockIdx.x == 3 && blockIdx.y == 0 && (idx) < 256) g_trace[ev][idx] = clock64(); } while (0)
+#define TR_SMID() do { unsigned s_; asm volatile("mov.u32 %0, %%smid;" : "=r"(s_)); if (blockIdx.x < 256 && blockIdx.y == 0) g_trace[21][blockIdx.x] = s_; } while (0)
 #define TR_GLOBAL(ev) do { long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); if (blockIdx.x < 256 && blockIdx.y == 0) g_trace[ev][blockIdx.x] = t_; } while (0)
 #else
 #define TR(ev, idx) do { } while (0)
 #define TR_GLOBAL(ev) do { } while (0)
+#define TR_SMID() do { } while (0)
 #endif
 
 constexpr int R = 512, DR = 64, K = R + DR;
@@ -205,9 +207,10 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_base_s;
-  if (tid == 0) { TR(13, 0); TR_GLOBAL(15); }
+  if (tid == 0) { TR(13, 0); TR_GLOBAL(15); TR_SMID(); }
   pdl_wait();  // the plan, the absorbed queries and the appended cache rows come from the kernel before this one
   const int4 pl = reinterpret_cast<const int4*>(plan)[part];
+  if (tid == 0) TR_GLOBAL(16);
 
   if (pl.y > pl.x) {
     if (warp == 4) {
@@ -227,6 +230,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
         if (pg_hi <= pg_lo) continue;
         {
           const uint32_t stage = acquire(g);
+          if (g == 0 && lane == 0) TR_GLOBAL(17);
           if (!*abort_flag && elect_one()) {
             mbar_arrive_expect_tx(bar(BAR_KV_FULL + stage), kChunks * kQTileBytes);
             const uint32_t dst = base + kOffStage + stage * kStageBytes;
@@ -292,6 +296,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
             const int stage = g % kStages, use = g / kStages;
             mbar_wait(bar(BAR_KV_FULL + stage), use & 1, abort_flag, dev_status);
             TR(1, g);
+            if (lane == 0) { if (n == 0) TR_GLOBAL(18); TR_GLOBAL(19); }
             if (n > 0) mbar_wait(bar(BAR_S_FREE), (n - 1) & 1, abort_flag, dev_status);
             TR(2, g);
             tc_fence_after();
@@ -481,7 +486,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
         // that its first QK^T runs while this segment's result is written out.
         const int b_next = next_segment(b);
         if (b_next <= pl.w) stage_queries();
-        if (tid == 0) TR(12, g);
+        if (tid == 0) { TR(12, g); TR_GLOBAL(20); }
         const int n_last = n - 1;
         mbar_wait(bar(BAR_PV_DONE0 + (n_last & 1)), (n_last >> 1) & 1, abort_flag, dev_status);
         tc_fence_after();
@@ -538,7 +543,7 @@ static PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
 
 #ifdef TRANSMLA_TRACE
 extern "C" int transmla_trace_dump(long long* host) {
-  return static_cast<int>(cudaMemcpyFromSymbol(host, sm100::g_trace, sizeof(long long) * 16 * 256));
+  return static_cast<int>(cudaMemcpyFromSymbol(host, sm100::g_trace, sizeof(long long) * 24 * 256));
 }
 #endif
 
