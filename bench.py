@@ -233,7 +233,8 @@ def run_ours(args, name, shape, seqlens, seed):
     ms_total = e0.elapsed_time(e1)
     clocks = sampler.stop(t0, t1) if sampler else None
     kernel_ms = statistics.mean(a.elapsed_time(b_) for a, b_ in kev.values())
-    assert int(status.item()) == 0, 'device status word set'
+    word = int(status.item())
+    assert word == 0, f'device status word {word:#x} after the timed steps'
 
     # end to end through the host-buffer entry point: pinned host inputs, result read back every step
     staging = torch.empty(binding.transmla_step_staging_bytes(params), dtype=torch.uint8, device='cuda')
@@ -244,9 +245,10 @@ def run_ours(args, name, shape, seqlens, seed):
     h_lse = torch.empty(B, S, H, dtype=torch.float32).pin_memory()
 
     def host_step(i):
-        return binding.transmla_decode_step_host(params, h['x'], h['q_nope'], h['q_pe'], h['page_table'], h['seqlens'],
+        word = binding.transmla_decode_step_host(params, h['x'], h['q_nope'], h['q_pe'], h['page_table'], h['seqlens'],
                                                  *weights[i % n_w], caches[i % n_copies], staging,
                                                  ws, h_out, h_lse, stream)
+        assert word == 0, f'device status word {word:#x} in host step {i}'
     for i in range(3):
         host_step(i)
     barrier()

@@ -51,7 +51,8 @@ typedef enum {
 /* page-equivalents charged to a partition for every sequence it opens (split plan) */
 #define TRANSMLA_SEGMENT_COST_PAGES 2
 
-/* bits of the device status word */
+/* bits of the device status word; when TRANSMLA_DEV_TIMEOUT is set, bits 8 and up tell which of the kernel's
+ * internal waits were still pending (diagnostic only, no stable meaning) */
 #define TRANSMLA_DEV_BAD_PAGE 1
 #define TRANSMLA_DEV_TIMEOUT 2
 
@@ -68,7 +69,12 @@ typedef struct {
   int32_t max_pages_per_seq; /* row stride of page_table */
   int32_t batch;             /* B */
   int32_t num_partitions;    /* G: how many pieces the batch's pages are split into; 0 = library chooses
-                                (SMs / row blocks, at most batch * max_pages_per_seq / 4) */
+                                (SMs / row blocks, at most batch * max_pages_per_seq / 4).  With an explicit G
+                                every partition handles exactly the page range of the plan and a rerun gives
+                                the same bits.  With 0, r = 512, dR = 64 and at least 8 partitions per
+                                sequence, the CTAs that share a sequence take its pages from a counter as they
+                                go (a CTA on a faster SM gets more): which pages meet in which partial then
+                                depends on timing, and results can differ in the last fp32 bits between runs */
   float softmax_scale;       /* 1/sqrt(dn + dR) for MLA (Eq. 9), 1/sqrt(d) for a lifted GQA layer (Eq. 13) */
   float rope_theta;          /* RoPE base, 10000 in Eq. 1 */
 } transmla_params_t;
@@ -79,8 +85,10 @@ typedef struct {
 /* Byte offsets of the regions inside the workspace that carries results from
  * transmla_mla_decode to transmla_mla_combine.  All regions are written by transmla_mla_decode.
  *   q_hat       bf16  [B, S, H, r+dR]   absorbed queries (Eq. 9 right, first line)
- *   cum_pages   int32 [3B+1]            [0..B]: slot prefix sums (below); [B+1..3B]: per sequence the first and
- *                                       last partition that holds pages of it (0, -1 for an empty sequence).
+ *   cum_pages   int32 [3B+1 + RB*B]     [0..B]: slot prefix sums (below); [B+1..3B]: per sequence the first and
+ *                                       last partition that holds pages of it (0, -1 for an empty sequence);
+ *                                       then one page counter per block of 32 query rows (RB = ceil(S*H/32)
+ *                                       of them) and sequence, used when pages are handed out at run time.
  *                                       Prefix sums: a sequence with n_b = ceil(L_b/P) > 0 pages owns
  *                                       TRANSMLA_SEGMENT_COST_PAGES virtual slots followed by its n_b page
  *                                       slots; cum[b] = number of slots before sequence b

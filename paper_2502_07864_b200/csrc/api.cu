@@ -116,7 +116,7 @@ transmla_status_t transmla_workspace_layout(const transmla_params_t* p, transmla
   out->num_partitions = G;
   out->num_slots = static_cast<int32_t>(slots);
   out->q_hat_offset = off;       off = round_up(off + B * SH * K * sizeof(__nv_bfloat16), kAlign);
-  out->cum_pages_offset = off;   off = round_up(off + (3 * B + 1) * sizeof(int32_t), kAlign);
+  out->cum_pages_offset = off;   off = round_up(off + (3 * B + 1 + (SH + kRowBlock - 1) / kRowBlock * B) * sizeof(int32_t), kAlign);
   out->plan_offset = off;        off = round_up(off + static_cast<size_t>(G) * 4 * sizeof(int32_t), kAlign);
   out->partial_o_offset = off;   off = round_up(off + slots * SH * p->kv_lora_rank * sizeof(float), kAlign);
   out->partial_lse_offset = off; off = round_up(off + slots * SH * sizeof(float), kAlign);

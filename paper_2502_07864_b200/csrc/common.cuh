@@ -11,6 +11,10 @@ namespace transmla {
 constexpr int kPage = 64;       // tokens per cache page (P)
 constexpr int kRowBlock = 32;   // query rows (s*H + h) one CTA works on
 constexpr int kSegCost = TRANSMLA_SEGMENT_COST_PAGES;  // virtual slots in front of every non-empty sequence
+// Dynamic page claims of the split-KV kernel (r = 512, dR = 64, partition count chosen by the library): the CTAs
+// whose partitions hold pages of a sequence take that sequence's pages one by one from a counter instead of
+// keeping to the plan's ranges, so a CTA on a faster SM ends up with more pages.  The counters next[rb][b] (one per
+// block of 32 query rows and sequence) sit behind the plan's prefix sums and partition ranges.
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
@@ -84,16 +88,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait.  Returns at once when the CTA has already given up.
+// Bounded wait.  Returns at once when the CTA has already given up.  For diagnosis, bit 8 + i of the status word
+// is set for every barrier slot i (position within its 256-byte block) on which a wait was still pending when the
+// CTA gave up; the first of them is the one whose limit expired.
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* dev_status) {
   if (*abort_flag) return;
   if (mbar_try_wait(bar, parity)) return;
   const long long t0 = clock64();
   while (!mbar_try_wait(bar, parity)) {
-    if (*abort_flag) return;
-    if (clock64() - t0 > kWaitCycles) {
+    const bool expired = clock64() - t0 > kWaitCycles;
+    if (expired || *abort_flag) {
       *abort_flag = 1;
-      set_status(dev_status, TRANSMLA_DEV_TIMEOUT);
+      set_status(dev_status, TRANSMLA_DEV_TIMEOUT | (1 << (8 + ((bar & 255u) >> 3))));
       return;
     }
   }
@@ -152,6 +158,7 @@ __device__ __forceinline__ unsigned long long trace_now() {
 #endif
 
 // Launchers (host).  Each enqueues on `stream` and returns the launch error, if any.
+bool dynamic_claims(const transmla_params_t& p, int G);  // whether the split-KV kernel hands pages out at run time
 cudaError_t launch_absorb_plan(const transmla_params_t& p, int G, const __nv_bfloat16* q_nope,
                                const __nv_bfloat16* q_pe, const __nv_bfloat16* w_uk, __nv_bfloat16* q_hat,
                                const int32_t* seqlens, int32_t* cum, int32_t* plan, cudaStream_t stream);

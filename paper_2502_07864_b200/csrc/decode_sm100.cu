@@ -34,11 +34,20 @@ namespace sm100 {
 __device__ long long g_trace[24][256];
 #define TR(ev, idx) do { if (blockIdx.x == 3 && blockIdx.y == 0 && (idx) < 256) g_trace[ev][idx] = clock64(); } while (0)
 #define TR_SMID() do { unsigned s_; asm volatile("mov.u32 %0, %%smid;" : "=r"(s_)); if (blockIdx.x < 256 && blockIdx.y == 0) g_trace[21][blockIdx.x] = s_; } while (0)
+#define TR_VAL(ev, v) do { if (blockIdx.x < 256 && blockIdx.y == 0) g_trace[ev][blockIdx.x] = (v); } while (0)
 #define TR_GLOBAL(ev) do { long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); if (blockIdx.x < 256 && blockIdx.y == 0) g_trace[ev][blockIdx.x] = t_; } while (0)
 #else
 #define TR(ev, idx) do { } while (0)
 #define TR_GLOBAL(ev) do { } while (0)
 #define TR_SMID() do { } while (0)
+#define TR_VAL(ev, v) do { } while (0)
+#endif
+
+#ifdef TRANSMLA_DBG
+__device__ int g_dbg[256][16];
+#define DBG(i, v) do { dbg_s[i] = (v); } while (0)
+#else
+#define DBG(i, v) do { } while (0)
 #endif
 
 constexpr int R = 512, DR = 64, K = R + DR;
@@ -50,6 +59,8 @@ constexpr int kPBytes = kRowBlock * 128;              // 4096: P[32 rows][64 tok
 constexpr int kQTileBytes = kRowBlock * 128;          // 4096: one 64-column sub-tile of the 32 query rows
 constexpr int kThreads = 192;
 constexpr uint32_t kTmemCols = 512;
+constexpr int kMetaRing = 16;            // descriptions of the ring items in flight (a power of two >= 2 * kStages)
+enum { ITEM_QUERIES = 1, ITEM_PAGE = 2, ITEM_END = 3 };
 constexpr uint32_t kColQ = 0, kColS = 288, kColO = 352;  // tensor-memory column map: Q_hat, S, O^T (4 x 32)
 
 // shared-memory map (offsets from a 1024-byte aligned base)
@@ -57,12 +68,12 @@ constexpr int kOffStage = 0;
 constexpr int kOffP = kStages * kStageBytes;      // 2 buffers
 constexpr int kOffBar = kOffP + 2 * kPBytes;      // mbarriers (8 bytes each)
 constexpr int kOffMisc = kOffBar + 128;
-// misc: m_s[2][32] f32, alpha_s[2][32] f32, flag_s[2] i32, l_part[4][32] f32, inv_l[32] f32, tmem base, abort
-constexpr int kMiscBytes = 256 + 256 + 16 + 512 + 128 + 16;
+// misc: pmax_s[2][4][32] f32, alpha_s[32] f32, inv_l[32] f32, meta[16] int4, tmem base, abort, ring_done
+constexpr int kMiscBytes = 1024 + 128 + 128 + 16 * kMetaRing + 16;
 constexpr int kSmemBytes = kOffMisc + kMiscBytes + 1024;  // + slack for the 1024-byte alignment
 static_assert(kSmemBytes <= 232448, "shared memory budget");
 
-enum { BAR_KV_FULL = 0, BAR_KV_EMPTY = kStages, BAR_Q_READY = 2 * kStages, BAR_S_FULL, BAR_S_FREE, BAR_P_READY,
+enum { BAR_KV_FULL = 0, BAR_KV_EMPTY = kStages, BAR_Q_READY = 2 * kStages, BAR_S_FULL, BAR_S_FREE, BAR_P_READY0, BAR_P_READY1,
        BAR_PV_DONE0, BAR_PV_DONE1 };
 
 // ---------------------------------------------------------------------------------------------- PTX wrappers
@@ -165,22 +176,26 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
                     const int32_t* __restrict__ page_table, const int32_t* __restrict__ seqlens,
                     const int32_t* __restrict__ cum, const int32_t* __restrict__ plan, float* __restrict__ partial_o,
                     float* __restrict__ partial_lse, int32_t* dev_status, int S, int H, int num_pages, int max_pages,
-                    float scale_log2) {
+                    float scale_log2, int B, int dynamic, int32_t* __restrict__ next) {
   extern __shared__ unsigned char smem_unaligned[];
   const uint32_t raw = smem_u32(smem_unaligned);
   const uint32_t base = (raw + 1023u) & ~1023u;
   unsigned char* sm = smem_unaligned + (base - raw);
-  float* m_s = reinterpret_cast<float*>(sm + kOffMisc);            // [2][32]
-  float* alpha_s = m_s + 64;                                       // [2][32]
-  int* flag_s = reinterpret_cast<int*>(alpha_s + 64);              // [2] (+2 pad)
-  float* l_part = reinterpret_cast<float*>(flag_s + 4);            // [4][32]
-  float* inv_l = l_part + 128;                                     // [32]
-  uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(inv_l + 32);
+  float* pmax_s = reinterpret_cast<float*>(sm + kOffMisc);         // [2][4][32]: per page parity, warp, row
+  float* alpha_s = pmax_s + 256;                                   // [32]
+  float* inv_l = alpha_s + 32;                                     // [32]
+  int4* meta = reinterpret_cast<int4*>(inv_l + 32);                // [kMetaRing]: what each ring item is
+  uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(meta + kMetaRing);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_base_s + 1);
+  volatile int* ring_done = abort_flag + 1;
   auto bar = [&](int i) -> uint32_t { return base + kOffBar + 8 * i; };
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int part = blockIdx.x, rb = blockIdx.y;
+#ifdef TRANSMLA_DBG
+  __shared__ volatile int dbg_s[16];
+  if (tid < 16) dbg_s[tid] = -1;
+#endif
   const int SH = S * H;
   pdl_trigger();
   TRK_BEGIN(1);
@@ -192,10 +207,12 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
     mbar_init(bar(BAR_Q_READY), 128);
     mbar_init(bar(BAR_S_FULL), 1);
     mbar_init(bar(BAR_S_FREE), 128);
-    mbar_init(bar(BAR_P_READY), 128);
+    mbar_init(bar(BAR_P_READY0), 128);
+    mbar_init(bar(BAR_P_READY1), 128);
     mbar_init(bar(BAR_PV_DONE0), 1);
     mbar_init(bar(BAR_PV_DONE1), 1);
     *abort_flag = 0;
+    *ring_done = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
@@ -211,11 +228,13 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
   pdl_wait();  // the plan, the absorbed queries and the appended cache rows come from the kernel before this one
   const int4 pl = reinterpret_cast<const int4*>(plan)[part];
   if (tid == 0) TR_GLOBAL(16);
+  const bool has_home = pl.y > pl.x;
 
-  if (pl.y > pl.x) {
+  if (has_home) {
     if (warp == 4) {
       // ======================================================================== TMA producer
-      // The ring carries, per segment, one item with the 32 absorbed query rows followed by the segment's pages.
+      // The ring carries, per segment, one item with the 32 absorbed query rows followed by the segment's pages,
+      // and one closing item when the CTA has nothing more to do.  What an item is goes into `meta`.
       int g = 0;  // ring items issued by this CTA so far
       const uint64_t stream_policy = l2_evict_first_policy();
       auto acquire = [&](int gi) -> uint32_t {  // waits for the stage of ring item gi; returns its index
@@ -224,110 +243,180 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
         TR(0, gi);
         return stage;
       };
+      auto issue_queries = [&](int b, int slot_code) {
+        const uint32_t stage = acquire(g);
+        if (g == 0 && lane == 0) TR_GLOBAL(17);
+        if (!*abort_flag && elect_one()) {
+          meta[g & (kMetaRing - 1)] = make_int4(ITEM_QUERIES, b, slot_code, seqlens[b]);
+          mbar_arrive_expect_tx(bar(BAR_KV_FULL + stage), kChunks * kQTileBytes);
+          const uint32_t dst = base + kOffStage + stage * kStageBytes;
+#pragma unroll
+          for (int c = 0; c < kChunks; ++c)
+            tma_load_2d(dst + c * kQTileBytes, &q_map, c * 64, b * SH + rb * kRowBlock, bar(BAR_KV_FULL + stage));
+        }
+        __syncwarp();
+        ++g;
+      };
+      auto issue_page = [&](int b, int pj, bool first, bool last) {
+        int idx = page_table[static_cast<size_t>(b) * max_pages + pj];
+        const bool ok = idx >= 0 && idx < num_pages;
+        if (!ok) { if (lane == 0) set_status(dev_status, TRANSMLA_DEV_BAD_PAGE); idx = 0; }
+        DBG(0, g); DBG(1, pj); DBG(2, (first ? 1 : 0) | (last ? 2 : 0));
+        const uint32_t stage = acquire(g);
+        if (!*abort_flag && elect_one()) {
+          meta[g & (kMetaRing - 1)] = make_int4(ITEM_PAGE, pj, ok ? 1 : 0, (first ? 1 : 0) | (last ? 2 : 0));
+          mbar_arrive_expect_tx(bar(BAR_KV_FULL + stage), kStageBytes);
+          const uint32_t dst = base + kOffStage + stage * kStageBytes;
+#pragma unroll
+          for (int c = 0; c < kChunks; ++c)
+            tma_load_2d_hint(dst + c * kSubTileBytes, &cache_map, c * 64, idx * kPage, bar(BAR_KV_FULL + stage), stream_policy);
+        }
+        __syncwarp();
+        ++g;
+      };
+      // ---- the partition's sequences in turn
       for (int b = pl.z; b <= pl.w; ++b) {
-        const int c0 = cum[b] + kSegCost;  // slot of page 0 of sequence b
-        const int pg_lo = max(pl.x, c0) - c0, pg_hi = min(pl.y, cum[b + 1]) - c0;
+        const int c0s = cum[b] + kSegCost;  // slot of page 0 of sequence b
+        const int pg_lo = max(pl.x, c0s) - c0s, pg_hi = min(pl.y, cum[b + 1]) - c0s;
         if (pg_hi <= pg_lo) continue;
-        {
-          const uint32_t stage = acquire(g);
-          if (g == 0 && lane == 0) TR_GLOBAL(17);
-          if (!*abort_flag && elect_one()) {
-            mbar_arrive_expect_tx(bar(BAR_KV_FULL + stage), kChunks * kQTileBytes);
-            const uint32_t dst = base + kOffStage + stage * kStageBytes;
-#pragma unroll
-            for (int c = 0; c < kChunks; ++c)
-              tma_load_2d(dst + c * kQTileBytes, &q_map, c * 64, b * SH + rb * kRowBlock, bar(BAR_KV_FULL + stage));
-          }
-          __syncwarp();
-          ++g;
+        if (!dynamic) {  // exactly the plan's range
+          issue_queries(b, part + b);
+          for (int pj = pg_lo; pj < pg_hi; ++pj) issue_page(b, pj, pj == pg_lo, pj == pg_hi - 1);
+          continue;
         }
-        for (int pj = pg_lo; pj < pg_hi; ++pj, ++g) {
-          int idx = page_table[static_cast<size_t>(b) * max_pages + pj];
-          if (idx < 0 || idx >= num_pages) { if (lane == 0) set_status(dev_status, TRANSMLA_DEV_BAD_PAGE); idx = 0; }
-          const uint32_t stage = acquire(g);
-          if (!*abort_flag && elect_one()) {
-            mbar_arrive_expect_tx(bar(BAR_KV_FULL + stage), kStageBytes);
-            const uint32_t dst = base + kOffStage + stage * kStageBytes;
-#pragma unroll
-            for (int c = 0; c < kChunks; ++c)
-              tma_load_2d_hint(dst + c * kSubTileBytes, &cache_map, c * 64, idx * kPage, bar(BAR_KV_FULL + stage), stream_policy);
-          }
-          __syncwarp();
+        // Pages of sequence b from its counter until it runs dry.  Three are claimed in one go (one atomic
+        // instruction, lanes 0..2) so that the stages fill at once.  After that the next two page numbers are
+        // always in hand and the claim behind them is in flight while a page waits for its stage, which keeps the
+        // counter's round trip off the critical path and tells at issue time whether a page is the segment's
+        // last one: it is exactly when the claim behind it is past the end (claims only grow).
+        const int n_b = cum[b + 1] - c0s;
+        int32_t* counter = next + static_cast<size_t>(rb) * B + b;
+        int head = 0x7fffffff;
+        if (lane < kStages) head = atomicAdd(counter, 1);
+        int c0 = __shfl_sync(0xffffffffu, head, 0), c1 = __shfl_sync(0xffffffffu, head, 1), c2 = __shfl_sync(0xffffffffu, head, 2);
+        { int t; if (c0 > c1) { t = c0; c0 = c1; c1 = t; } if (c1 > c2) { t = c1; c1 = c2; c2 = t; } if (c0 > c1) { t = c0; c0 = c1; c1 = t; } }
+        if (c0 >= n_b) {  // the others have taken everything: the combine still expects a partial from this slot
+          if (rb * kRowBlock + lane < SH) partial_lse[static_cast<size_t>(part + b) * SH + rb * kRowBlock + lane] = -INFINITY;
+          continue;
         }
+        issue_queries(b, part + b);
+        bool first = true;
+        while (c0 < n_b) {
+          int pend = 0x7fffffff;
+          const bool ahead = c2 < n_b;
+          if (ahead && lane == 0) pend = atomicAdd(counter, 1);
+          issue_page(b, c0, first, c1 >= n_b);
+          first = false;
+          c0 = c1;
+          c1 = c2;
+          c2 = ahead ? __shfl_sync(0xffffffffu, pend, 0) : 0x7fffffff;
+        }
+      }
+      if (lane == 0) TR_VAL(22, g);
+      {  // closing item
+        const uint32_t stage = acquire(g);
+        if (elect_one()) {
+          meta[g & (kMetaRing - 1)] = make_int4(ITEM_END, 0, 0, 0);
+          mbar_arrive(bar(BAR_KV_FULL + stage));
+        }
+        __syncwarp();
       }
     } else if (warp == 5) {
       // ======================================================================== MMA issuer
-      {
-        constexpr uint32_t idesc_qk = instr_desc(kPage, false);
-        constexpr uint32_t idesc_pv = instr_desc(kRowBlock, true);
-        int g = 0, n = 0, seg = 0;  // ring items, pages, segments handled so far
-        auto issue_pv = [&](int gr, int gp, bool first_of_segment) {  // O^T += C^T P^T for page gp held in ring item gr
-          const int stage = gr % kStages;
-          mbar_wait(bar(BAR_P_READY), gp & 1, abort_flag, dev_status);
-          TR(4, gr);
-          tc_fence_after();
-          const uint64_t a0 = smem_desc(base + kOffStage + stage * kStageBytes, kSubTileBytes, 1024);
-          const uint64_t b0 = smem_desc(base + kOffP + (gp & 1) * kPBytes, 16, 1024);
-          const uint32_t acc0 = first_of_segment ? 0u : 1u;
+      // Follows the ring: skips query items (the softmax warps move them to tensor memory and report through
+      // Q_READY, which also tells when the ring has ended), runs QK^T for a page as soon as it has landed and
+      // the PV of the page before it one step later.
+      constexpr uint32_t idesc_qk = instr_desc(kPage, false);
+      constexpr uint32_t idesc_pv = instr_desc(kRowBlock, true);
+      int g = 0, n = 0, seg = 0;  // ring items, pages, segments handled so far
+      auto issue_pv = [&](int gr, int gp, bool first_of_segment) {  // O^T += C^T P^T for page gp held in ring item gr
+        const int stage = gr % kStages;
+        // One barrier per P buffer: the softmax warps can run a page ahead of this warp (S is ready before the PV
+        // of the page before it is issued), and with a single barrier two of its phases could complete before this
+        // wait looks at the first.  Per buffer the next phase needs the PV issued below to have completed.
+        mbar_wait(bar(BAR_P_READY0 + (gp & 1)), (gp >> 1) & 1, abort_flag, dev_status);
+        TR(4, gr);
+        tc_fence_after();
+        const uint64_t a0 = smem_desc(base + kOffStage + stage * kStageBytes, kSubTileBytes, 1024);
+        const uint64_t b0 = smem_desc(base + kOffP + (gp & 1) * kPBytes, 16, 1024);
+        const uint32_t acc0 = first_of_segment ? 0u : 1u;
 #pragma unroll
-          for (int kk = 0; kk < 4; ++kk) {
+        for (int kk = 0; kk < 4; ++kk) {
 #pragma unroll
-            for (int t = 0; t < 4; ++t) {
-              if (elect_one())
-                mma_ss(tmem + kColO + t * 32, desc_advance(a0, (2 * t) * kSubTileBytes + kk * 2048),
-                       desc_advance(b0, kk * 32), idesc_pv, kk == 0 ? acc0 : 1u);
-            }
+          for (int t = 0; t < 4; ++t) {
+            if (elect_one())
+              mma_ss(tmem + kColO + t * 32, desc_advance(a0, (2 * t) * kSubTileBytes + kk * 2048),
+                     desc_advance(b0, kk * 32), idesc_pv, kk == 0 ? acc0 : 1u);
           }
-          if (elect_one()) {
-            tc_commit(bar(BAR_KV_EMPTY + stage));
-            tc_commit(bar(BAR_PV_DONE0 + (gp & 1)));
-          }
-          __syncwarp();
-          TR(5, gr);
-        };
-        for (int b = pl.z; b <= pl.w; ++b) {
-          const int c0 = cum[b] + kSegCost;  // slot of page 0 of sequence b
-          const int pg_lo = max(pl.x, c0) - c0, pg_hi = min(pl.y, cum[b + 1]) - c0;
-          if (pg_hi <= pg_lo) continue;
-          ++g;  // the segment's query item is consumed by the softmax warps
-          mbar_wait(bar(BAR_Q_READY), seg & 1, abort_flag, dev_status);
-          ++seg;
-          for (int pj = pg_lo; pj < pg_hi; ++pj, ++g, ++n) {
-            const int stage = g % kStages, use = g / kStages;
-            mbar_wait(bar(BAR_KV_FULL + stage), use & 1, abort_flag, dev_status);
-            TR(1, g);
-            if (lane == 0) { if (n == 0) TR_GLOBAL(18); TR_GLOBAL(19); }
-            if (n > 0) mbar_wait(bar(BAR_S_FREE), (n - 1) & 1, abort_flag, dev_status);
-            TR(2, g);
-            tc_fence_after();
-            const uint64_t k0 = smem_desc(base + kOffStage + stage * kStageBytes, 16, 1024);
-#pragma unroll
-            for (int c = 0; c < kChunks; ++c) {
-#pragma unroll
-              for (int kk = 0; kk < 4; ++kk) {
-                if (elect_one())
-                  mma_ts(tmem + kColS, tmem + kColQ + c * 32 + kk * 8, desc_advance(k0, c * kSubTileBytes + kk * 32),
-                         idesc_qk, (c | kk) ? 1u : 0u);
-              }
-            }
-            if (elect_one()) tc_commit(bar(BAR_S_FULL));
-            __syncwarp();
-            TR(3, g);
-            if (pj > pg_lo) issue_pv(g - 1, n - 1, pj - 1 == pg_lo);
-          }
-          issue_pv(g - 1, n - 1, pg_hi - 1 == pg_lo);
         }
+        if (elect_one()) {
+          tc_commit(bar(BAR_KV_EMPTY + stage));
+          tc_commit(bar(BAR_PV_DONE0 + (gp & 1)));
+        }
+        __syncwarp();
+        TR(5, gr);
+      };
+      while (true) {
+        // a segment begins (or the ring ends): the softmax warps say which
+        mbar_wait(bar(BAR_Q_READY), seg & 1, abort_flag, dev_status);
+        ++seg;
+        if (__any_sync(0xffffffffu, *abort_flag != 0) || *ring_done != 0) break;
+        ++g;  // the query item
+        bool pending = false, pending_first = false;
+        while (true) {
+          const int stage = g % kStages, use = g / kStages;
+          mbar_wait(bar(BAR_KV_FULL + stage), use & 1, abort_flag, dev_status);
+          const int4 m = meta[g & (kMetaRing - 1)];
+          DBG(4, g); DBG(5, n); DBG(6, seg); DBG(7, m.w | (m.x << 8));
+          TR(1, g);
+          if (lane == 0) { if (n == 0) TR_GLOBAL(18); TR_GLOBAL(19); }
+          if (n > 0) mbar_wait(bar(BAR_S_FREE), (n - 1) & 1, abort_flag, dev_status);
+          TR(2, g);
+          tc_fence_after();
+          const uint64_t k0 = smem_desc(base + kOffStage + stage * kStageBytes, 16, 1024);
+#pragma unroll
+          for (int c = 0; c < kChunks; ++c) {
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+              if (elect_one())
+                mma_ts(tmem + kColS, tmem + kColQ + c * 32 + kk * 8, desc_advance(k0, c * kSubTileBytes + kk * 32),
+                       idesc_qk, (c | kk) ? 1u : 0u);
+            }
+          }
+          if (elect_one()) tc_commit(bar(BAR_S_FULL));
+          __syncwarp();
+          TR(3, g);
+          if (pending) issue_pv(g - 1, n - 1, pending_first);
+          pending = true;
+          pending_first = (m.w & 1) != 0;
+          ++g; ++n;
+          if ((m.w & 2) != 0 || m.x != ITEM_PAGE || __any_sync(0xffffffffu, *abort_flag != 0)) break;
+        }
+        issue_pv(g - 1, n - 1, pending_first);
       }
     } else {
       // ======================================================================== softmax + epilogue (warps 0-3)
       const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
       const int my_row = rb * kRowBlock + lane;  // query row of this thread (same in all four replicas)
       int g = 0, n = 0;  // ring items and pages handled so far
-      // Q_hat rows of the next ring item: shared memory (swizzled sub-tiles of 32 rows x 128 bytes) -> this
-      // warp's replica in tensor memory, 32 columns (64 elements) at a time; then the stage is handed back.
-      auto stage_queries = [&]() {
+      // Looks at ring item g.  Queries: moves the 32 rows from shared memory (swizzled sub-tiles of 32 rows x
+      // 128 bytes) to this warp's replica in tensor memory, 32 columns (64 elements) at a time, hands the stage
+      // back and returns the item's description.  Closing item: marks the ring as ended.  Either way the MMA
+      // warp is told through Q_READY.  All 128 threads take the same path (the description is the same for all).
+      auto open_segment = [&]() -> int4 {
         const int stage = g % kStages, use = g / kStages;
         mbar_wait(bar(BAR_KV_FULL + stage), use & 1, abort_flag, dev_status);
+        int4 m = meta[g & (kMetaRing - 1)];
+        int aborted;
+        asm volatile("{\n.reg .pred p, q;\nsetp.ne.b32 q, %1, 0;\nbar.red.or.pred p, 1, 128, q;\nselp.s32 %0, 1, 0, p;\n}"
+                     : "=r"(aborted) : "r"(*abort_flag) : "memory");
+        if (aborted || m.x != ITEM_QUERIES) {
+          m.x = ITEM_END;
+          if (tid == 0) *ring_done = 1;
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+          mbar_arrive(bar(BAR_Q_READY));
+          return m;
+        }
         const unsigned char* qrow = sm + kOffStage + stage * kStageBytes + lane * 128;
 #pragma unroll 1
         for (int c = 0; c < kChunks; ++c) {
@@ -345,31 +434,27 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (tid == 0) { mbar_arrive(bar(BAR_KV_EMPTY + stage)); TR(11, g); }
         ++g;
+        return m;
       };
-      auto next_segment = [&](int b) -> int {  // first sequence after b that has pages in this partition, or pl.w + 1
-        for (++b; b <= pl.w; ++b) {
-          const int c0 = cum[b] + kSegCost;  // slot of page 0 of sequence b
-          if (min(pl.y, cum[b + 1]) > max(pl.x, c0)) break;
-        }
-        return b;
-      };
-      int b = next_segment(pl.z - 1);
-      if (b <= pl.w) stage_queries();
-      while (b <= pl.w) {
-        const int c0 = cum[b] + kSegCost;  // slot of page 0 of sequence b
-        const int pg_lo = max(pl.x, c0) - c0, pg_hi = min(pl.y, cum[b + 1]) - c0;
-        const int L = seqlens[b];
-        const int slot = part + b;
+      int4 seg_meta = open_segment();
+      while (seg_meta.x == ITEM_QUERIES) {
+        const int L = seg_meta.w;
+        float* o_rows = partial_o + (static_cast<size_t>(seg_meta.z) * SH + rb * kRowBlock) * R;
+        float* lse_rows = partial_lse + static_cast<size_t>(seg_meta.z) * SH + rb * kRowBlock;
         const int n_vis = my_row < SH ? L - (S - 1 - my_row / H) : 0;
 
         float m_used = -INFINITY, l_run = 0.f;
-        for (int pj = pg_lo; pj < pg_hi; ++pj, ++g, ++n) {
+        bool more = true;
+        while (more) {
           const int stage = g % kStages;
-          const int idx = page_table[static_cast<size_t>(b) * max_pages + pj];
-          const bool page_ok = idx >= 0 && idx < num_pages;
+          mbar_wait(bar(BAR_KV_FULL + stage), (g / kStages) & 1, abort_flag, dev_status);
+          const int4 pm = meta[g & (kMetaRing - 1)];
+          if (tid == 0) { DBG(8, g); DBG(9, n); DBG(10, pm.w | (pm.x << 8)); DBG(11, pm.y); }
+          const int pj = pm.y;
+          const bool page_ok = pm.z != 0;
           const int tok_end = page_ok ? n_vis - pj * kPage : 0;           // tokens [0, tok_end) of the page are visible
           const int valid = page_ok ? min(kPage, L - pj * kPage) : 0;      // rows [valid, 64) must read as zero
-          const bool first = pj == pg_lo;
+          const bool first = (pm.w & 1) != 0;
           const int buf = n & 1;
 
           if (tid == 0) TR(6, g);
@@ -377,49 +462,41 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
           if (tid == 0) TR(7, g);
           tc_fence_after();
           uint32_t sq[16];  // this warp's 16 tokens of its row
-          float rowmax = -INFINITY;
-          if (warp == 0) {
-            uint32_t sv[64];
-            tmem_ld32(tmem + lane_base + kColS, sv);
-            tmem_ld32(tmem + lane_base + kColS + 32, sv + 32);
-            tc_wait_ld();
-#pragma unroll
-            for (int j = 0; j < 64; ++j)
-              rowmax = fmaxf(rowmax, j < tok_end ? __uint_as_float(sv[j]) * scale_log2 : -INFINITY);
-#pragma unroll
-            for (int j = 0; j < 16; ++j) sq[j] = sv[j];
-          } else {
-            tmem_ld16(tmem + lane_base + kColS + warp * 16, sq);
-            tc_wait_ld();
-          }
+          tmem_ld16(tmem + lane_base + kColS + warp * 16, sq);
+          tc_wait_ld();
           tc_fence_before();
           mbar_arrive(bar(BAR_S_FREE));
           if (tid == 0) TR(8, g);
-
-          if (warp == 0) {
-            // Lazy rescale: the reference maximum only moves when some row's new maximum exceeds it by 2^8.
-            float alpha = 1.f;
-            bool need = false;
-            if (first) {
-              m_used = rowmax;
-            } else {
-              need = rowmax > m_used + 8.f;
-            }
-            const bool any = __any_sync(0xffffffffu, need);
-            if (any) {
+          {
+            float pmax = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+              pmax = fmaxf(pmax, warp * 16 + j < tok_end ? __uint_as_float(sq[j]) * scale_log2 : -INFINITY);
+            pmax_s[(buf * 4 + warp) * 32 + lane] = pmax;
+          }
+          // one barrier per page: the row maxima meet, and all 128 threads learn together whether the CTA gave up
+          int aborted;
+          asm volatile("{\n.reg .pred p, q;\nsetp.ne.b32 q, %1, 0;\nbar.red.or.pred p, 1, 128, q;\nselp.s32 %0, 1, 0, p;\n}"
+                       : "=r"(aborted) : "r"(*abort_flag) : "memory");
+          more = (pm.w & 2) == 0 && pm.x == ITEM_PAGE && !aborted;
+          const float rowmax = fmaxf(fmaxf(pmax_s[(buf * 4 + 0) * 32 + lane], pmax_s[(buf * 4 + 1) * 32 + lane]),
+                                     fmaxf(pmax_s[(buf * 4 + 2) * 32 + lane], pmax_s[(buf * 4 + 3) * 32 + lane]));
+          // Lazy rescale: the reference maximum only moves when some row's new maximum exceeds it by 2^8.  Every
+          // warp holds all 32 rows, so the four warps take the same decision without talking to each other.
+          float alpha = 1.f;
+          bool rescale = false;
+          if (first) {
+            m_used = rowmax;
+          } else {
+            rescale = __any_sync(0xffffffffu, rowmax > m_used + 8.f);
+            if (rescale) {
               const float m_new = fmaxf(m_used, rowmax);
               alpha = (m_new == -INFINITY) ? 1.f : exp2f(m_used - m_new);
               m_used = m_new;
+              l_run *= alpha;
             }
-            m_s[buf * 32 + lane] = m_used;
-            alpha_s[buf * 32 + lane] = alpha;
-            if (lane == 0) flag_s[buf] = any ? 1 : 0;
           }
-          asm volatile("bar.sync 1, 128;" ::: "memory");
-          const float m_ref = m_s[buf * 32 + lane];
-          const bool rescale = flag_s[buf] != 0;
-          if (rescale) l_run *= alpha_s[buf * 32 + lane];
-          m_used = m_ref;
+          const float m_ref = m_used;
 
           // ---- probabilities of tokens 16*warp .. 16*warp+15
           uint32_t pk[8];
@@ -434,7 +511,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
           }
           l_run += psum;
 
-          // ---- P buffer `buf` is free once PV of CTA page g-2 is done
+          // ---- P buffer `buf` is free once PV of CTA page n-2 is done
           if (n >= 2) mbar_wait(bar(BAR_PV_DONE0 + buf), ((n >> 1) - 1) & 1, abort_flag, dev_status);
           {
             unsigned char* prow = sm + kOffP + buf * kPBytes + lane * 128;
@@ -453,6 +530,8 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
           }
           // ---- rescale O^T by alpha (columns = query rows) once the previous PV has landed
           if (rescale) {
+            if (warp == 0) alpha_s[lane] = alpha;
+            asm volatile("bar.sync 1, 128;" ::: "memory");  // a later rescale is at least one page barrier away
             if (n >= 1) mbar_wait(bar(BAR_PV_DONE0 + ((n - 1) & 1)), ((n - 1) >> 1) & 1, abort_flag, dev_status);
             tc_fence_after();
 #pragma unroll 1
@@ -461,36 +540,38 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
               tmem_ld32(tmem + lane_base + kColO + t * 32, ov);
               tc_wait_ld();
 #pragma unroll
-              for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * alpha_s[buf * 32 + j]);
+              for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * alpha_s[j]);
               tmem_st32(tmem + lane_base + kColO + t * 32, ov);
             }
             tc_wait_st();
           }
           fence_proxy_async();
           tc_fence_before();
-          mbar_arrive(bar(BAR_P_READY));
+          mbar_arrive(bar(BAR_P_READY0 + buf));
           if (tid == 0) TR(9, g);
+          ++g; ++n;
         }
 
-        // ---- epilogue of the segment: wait for the last PV, normalise, store O (transposed back) and lse
+        // ---- epilogue of the segment: wait for the last PV, normalise, store O (transposed back) and lse.
+        // The row sums meet in the half of pmax_s that the last page did not use (its readers are behind the
+        // last page's barrier; the next page writes it only after the barrier at the end of this epilogue).
+        float* l_part = pmax_s + (n & 1) * 128;
         l_part[warp * 32 + lane] = l_run;
         asm volatile("bar.sync 1, 128;" ::: "memory");
         const float l_tot = l_part[lane] + l_part[32 + lane] + l_part[64 + lane] + l_part[96 + lane];
         if (warp == 0) {
           inv_l[lane] = l_tot > 0.f ? 1.f / l_tot : 0.f;
-          if (my_row < SH)
-            partial_lse[static_cast<size_t>(slot) * SH + my_row] = l_tot > 0.f ? (m_used + log2f(l_tot)) * kLn2 : -INFINITY;
+          if (my_row < SH) lse_rows[lane] = l_tot > 0.f ? (m_used + log2f(l_tot)) * kLn2 : -INFINITY;
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
         // The queries of the next segment go to tensor memory now (every QK^T of this segment has completed), so
         // that its first QK^T runs while this segment's result is written out.
-        const int b_next = next_segment(b);
-        if (b_next <= pl.w) stage_queries();
+        seg_meta = open_segment();
         if (tid == 0) { TR(12, g); TR_GLOBAL(20); }
         const int n_last = n - 1;
         mbar_wait(bar(BAR_PV_DONE0 + (n_last & 1)), (n_last >> 1) & 1, abort_flag, dev_status);
         tc_fence_after();
-        float* dst = partial_o + (static_cast<size_t>(slot) * SH + rb * kRowBlock) * R + warp * 32 + lane;
+        float* dst = o_rows + warp * 32 + lane;
 #pragma unroll 1
         for (int t = 0; t < 4; t += 2) {  // two 128-row tiles per round trip to tensor memory
           uint32_t ov[64];
@@ -507,14 +588,17 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
           }
         }
         tc_fence_before();
-        asm volatile("bar.sync 1, 128;" ::: "memory");  // inv_l / l_part are reused by the next segment
+        asm volatile("bar.sync 1, 128;" ::: "memory");  // inv_l and the row sums are reused by the next segment
         if (tid == 0) TR(14, g);
-        b = b_next;
       }
     }
   }
 
   if (tid == 0) { TR(13, 1); TR_GLOBAL(10); }
+#ifdef TRANSMLA_DBG
+  __syncthreads();
+  if (*abort_flag && tid < 16 && blockIdx.x < 256 && blockIdx.y == 0) g_dbg[blockIdx.x][tid] = dbg_s[tid];
+#endif
   TRK_END(1);
   // ---- teardown: everyone arrives, tensor memory is returned
   tc_fence_before();
@@ -541,6 +625,9 @@ static PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
 
 }  // namespace sm100
 
+#ifdef TRANSMLA_DBG
+extern "C" int transmla_dbg_dump(int* host) { return static_cast<int>(cudaMemcpyFromSymbol(host, sm100::g_dbg, sizeof(int) * 256 * 16)); }
+#endif
 #ifdef TRANSMLA_TRACE
 extern "C" int transmla_trace_dump(long long* host) {
   return static_cast<int>(cudaMemcpyFromSymbol(host, sm100::g_trace, sizeof(long long) * 24 * 256));
@@ -548,6 +635,14 @@ extern "C" int transmla_trace_dump(long long* host) {
 #endif
 
 bool decode_sm100_supported(const transmla_params_t& p) { return p.kv_lora_rank == sm100::R && p.qk_rope_dim == sm100::DR; }
+
+// Pages are handed out at run time only when the library chose the partition count itself (a caller who fixes the
+// count gets the plan's page ranges, and with them results that do not depend on timing) and only when a sequence
+// is shared by many CTAs: the CTAs of a partition that straddles two sequences finish the first sequence's pages
+// before they join the second, which costs more than the claims gain once sequences have only a few CTAs each.
+bool dynamic_claims(const transmla_params_t& p, int G) {
+  return p.num_partitions == 0 && decode_sm100_supported(p) && G >= 8 * p.batch;
+}
 
 cudaError_t launch_decode_sm100(const transmla_params_t& p, int G, const __nv_bfloat16* q_hat,
                                 const __nv_bfloat16* cache, const int32_t* page_table, const int32_t* seqlens,
@@ -583,9 +678,10 @@ cudaError_t launch_decode_sm100(const transmla_params_t& p, int G, const __nv_bf
     attr_set = true;
   }
   dim3 grid(G, (SH + kRowBlock - 1) / kRowBlock);
+  int32_t* next = const_cast<int32_t*>(cum) + 3 * p.batch + 1;  // page counters, zeroed by the plan
   return launch_pdl(decode_sm100_kernel, grid, dim3(kThreads), static_cast<size_t>(kSmemBytes), stream, map, qmap,
                     page_table, seqlens, cum, plan, partial_o, partial_lse, dev_status, p.q_len, p.num_heads,
-                    p.num_pages, p.max_pages_per_seq, p.softmax_scale * kLog2e);
+                    p.num_pages, p.max_pages_per_seq, p.softmax_scale * kLog2e, p.batch, dynamic_claims(p, G) ? 1 : 0, next);
 }
 
 }  // namespace transmla

@@ -60,7 +60,7 @@ __device__ __forceinline__ int seq_of_page(const int32_t* cum, int B, int x) {
   return lo - 1;
 }
 
-__device__ void plan_block(const int32_t* __restrict__ seqlens, int B, int G, int32_t* cum, int32_t* plan,
+__device__ void plan_block(const int32_t* __restrict__ seqlens, int B, int G, int RB, int32_t* cum, int32_t* plan,
                            unsigned char* smem_raw) {
   __shared__ int warp_sums[8];
   __shared__ int carry;
@@ -109,6 +109,10 @@ __device__ void plan_block(const int32_t* __restrict__ seqlens, int B, int G, in
     seq_parts[2 * b] = i_first;
     seq_parts[2 * b + 1] = i_last;
   }
+  // The page counters of the split-KV kernel start at zero.  Every earlier kernel of the stream has completed
+  // here (the dependency wait above), so nobody is still counting.
+  int32_t* next = cum + 3 * B + 1;
+  for (int i = tid; i < RB * B; i += 256) next[i] = 0;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -241,7 +245,7 @@ __global__ void __launch_bounds__(256) absorb_plan_kernel(const __nv_bfloat16* _
   if (static_cast<int>(blockIdx.x) < n_absorb) {
     absorb_block(q_nope, q_pe, w_uk, q_hat, B * S, H, dn, dR, r, blockIdx.x / r_tiles, blockIdx.x % r_tiles, smem_raw);
   } else {
-    plan_block(seqlens, B, G, cum, plan, smem_raw);
+    plan_block(seqlens, B, G, (S * H + kRowBlock - 1) / kRowBlock, cum, plan, smem_raw);
   }
 }
 
@@ -260,7 +264,7 @@ __global__ void __launch_bounds__(256) prologue_kernel(
   const int r_tiles = (r + 127) / 128;
   const int bid = static_cast<int>(blockIdx.x) - 1;
   if (bid < 0) {
-    plan_block(seqlens, B, G, cum, plan, smem_raw);
+    plan_block(seqlens, B, G, (S * H + kRowBlock - 1) / kRowBlock, cum, plan, smem_raw);
   } else if (bid < n_append) {
     append_block(x, w_dkv_kr, seqlens, -S, page_table, cache, dev_status, B, S, D, r, dR, num_pages, max_pages, theta,
                  bid, t_splits, smem_raw);

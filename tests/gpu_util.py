@@ -21,11 +21,18 @@ def to_dev(case):
     return {k: (v.cuda() if isinstance(v, torch.Tensor) else v) for k, v in case.items()}
 
 
-def gpu_decode(shape, case, scale, G=0, want_views=False):
-    """decode + combine through the C ABI on device tensors.  Returns out, lse, status word, views."""
+def gpu_decode(shape, case, scale, G=0, want_views=False, fixed_plan=False):
+    """decode + combine through the C ABI on device tensors.  Returns out, lse, status word, views.
+
+    G = 0 lets the library choose the partition count; it then also hands pages to CTAs dynamically, so
+    which pages end up in which partial depends on timing.  With ``fixed_plan`` the library's own count is
+    passed back explicitly, which pins every partition to the page range of the plan.
+    """
     B = case['seqlens'].numel()
     params = binding.make_params(shape, B, case['cache'].shape[0], case['page_table'].shape[1], scale,
                                  num_partitions=G)
+    if G == 0 and fixed_plan:
+        params.num_partitions = binding.transmla_workspace_layout(params).num_partitions
     ws, lay = binding.alloc_workspace(params)
     status = torch.zeros(1, dtype=torch.int32, device='cuda')
     out = torch.full((B, shape.S, shape.H, shape.dv), float('nan'), dtype=torch.bfloat16, device='cuda')

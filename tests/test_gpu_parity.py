@@ -25,7 +25,8 @@ def _lib():
 def _run_and_compare(shape, seqlens, seed, G=0, scale=None, nan_tails=True, check_internals=False):
     scale = scale if scale is not None else gu.mla_scale(shape)
     case = synth.make_decode_case(shape, seqlens, seed, nan_tails=nan_tails)
-    out, lse, status, views, lay = gu.gpu_decode(shape, gu.to_dev(case), scale, G=G, want_views=check_internals)
+    out, lse, status, views, lay = gu.gpu_decode(shape, gu.to_dev(case), scale, G=G, want_views=check_internals,
+                                                 fixed_plan=check_internals)
     assert status == 0
     want_out, want_lse = gu.oracle_decode(shape, case, scale)
     gu.assert_close(lifts.f64(out), want_out, f'out seqlens={seqlens} G={G}')
