@@ -314,3 +314,51 @@ def test_layer_decode_step(shape, seqlens, rq):
                                 dc['page_table'].numpy(), seqlens, scale, shape.r,
                                 w_dq=None if not rq else lifts.f64(lw['w_dq']))
     err, rel = gu.assert_close(lifts.f64(y), want, f'layer output rq={rq}')
+
+
+# ------------------------------------------------------------------ pages claimed at run time (G = 0, many CTAs per sequence)
+@pytest.mark.parametrize('seqlens', [[4096 + 17, 2100], [8192], [64 * 40, 64 * 41 + 1, 3000]])
+def test_dynamic_page_claims_match_the_oracle(seqlens):
+    # With G = 0 and at least 8 partitions per sequence the CTAs of a sequence take its pages from a counter, so
+    # the grouping of pages into partials depends on timing: what is unique is the combined result.
+    shape = synth.LLAMA2_7B
+    scale = gu.mla_scale(shape)
+    case = synth.make_decode_case(shape, seqlens, seed=23, nan_tails=True)
+    dev = gu.to_dev(case)
+    only = [(b, 0, h) for b in range(len(seqlens)) for h in (0, 5, 31)]
+    want, want_lse = gu.oracle_decode(shape, case, scale, only=only)
+    idx = tuple(np.array(only).T)
+    for _ in range(3):
+        out, lse, status, _, lay = gu.gpu_decode(shape, dev, scale, G=0)
+        assert status == 0 and lay.num_partitions >= 8 * len(seqlens)
+        gu.assert_close(lifts.f64(out)[idx], want[idx], f'dynamic claims {seqlens}')
+        gu.assert_lse_close(lifts.f64(lse)[idx], want_lse[idx], 'dynamic claims lse')
+
+
+@pytest.mark.parametrize('G', [0, 37])
+def test_many_serialized_launches_never_time_out(G):
+    # Launches bracketed by events start all CTAs at once with cold instruction caches, which is when the softmax
+    # warps can get a whole page ahead of the MMA warp; every bounded wait must still be satisfied.
+    shape = synth.LLAMA2_7B
+    seqlens = [1024] * 4
+    case = gu.to_dev(synth.make_decode_case(shape, seqlens, seed=24))
+    B = len(seqlens)
+    params = binding.make_params(shape, B, case['cache'].shape[0], case['page_table'].shape[1], gu.mla_scale(shape),
+                                 num_partitions=G)
+    ws, lay = binding.alloc_workspace(params)
+    status = torch.zeros(1, dtype=torch.int32, device='cuda')
+    out = torch.empty(B, 1, shape.H, shape.dv, dtype=torch.bfloat16, device='cuda')
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    for e in evs:
+        e.record()
+    first = None
+    for i in range(3000):
+        binding.transmla_profile_decode_kernel(evs[0], evs[1])
+        binding.transmla_mla_decode(params, case['q_nope'], case['q_pe'], case['w_uk'], case['cache'], case['page_table'],
+                                    case['seqlens'], ws, status)
+        binding.transmla_mla_combine(params, ws, case['w_uv'], out, None, status)
+        if i == 0:
+            first = out.clone()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert (out.float() - first.float()).abs().max().item() <= 2e-2
