@@ -243,11 +243,11 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
         TR(0, gi);
         return stage;
       };
-      auto issue_queries = [&](int b, int slot_code) {
+      auto issue_queries = [&](int b, int slot_code, int L) {
         const uint32_t stage = acquire(g);
         if (g == 0 && lane == 0) TR_GLOBAL(17);
         if (!*abort_flag && elect_one()) {
-          meta[g & (kMetaRing - 1)] = make_int4(ITEM_QUERIES, b, slot_code, seqlens[b]);
+          meta[g & (kMetaRing - 1)] = make_int4(ITEM_QUERIES, b, slot_code, L);
           mbar_arrive_expect_tx(bar(BAR_KV_FULL + stage), kChunks * kQTileBytes);
           const uint32_t dst = base + kOffStage + stage * kStageBytes;
 #pragma unroll
@@ -275,12 +275,21 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
         ++g;
       };
       // ---- the partition's sequences in turn
+      // Page-table entries [lo, hi) of sequence b are asked into L1 ahead of their use (one 128-byte line per lane
+      // and round), so that the look-up in front of every page load does not cost a trip to L2.
+      auto prefetch_table = [&](int b, int lo, int hi) {
+        const int32_t* row = page_table + static_cast<size_t>(b) * max_pages;
+        for (int i = (lo & ~31) + lane * 32; i < hi; i += 32 * 32)
+          asm volatile("prefetch.global.L1 [%0];" ::"l"(row + max(i, lo)));
+      };
       for (int b = pl.z; b <= pl.w; ++b) {
-        const int c0s = cum[b] + kSegCost;  // slot of page 0 of sequence b
-        const int pg_lo = max(pl.x, c0s) - c0s, pg_hi = min(pl.y, cum[b + 1]) - c0s;
+        const int cb = cum[b], cb1 = cum[b + 1], L = seqlens[b];  // one round trip for the three of them
+        const int c0s = cb + kSegCost;  // slot of page 0 of sequence b
+        const int pg_lo = max(pl.x, c0s) - c0s, pg_hi = min(pl.y, cb1) - c0s;
         if (pg_hi <= pg_lo) continue;
         if (!dynamic) {  // exactly the plan's range
-          issue_queries(b, part + b);
+          prefetch_table(b, pg_lo, pg_hi);
+          issue_queries(b, part + b, L);
           for (int pj = pg_lo; pj < pg_hi; ++pj) issue_page(b, pj, pj == pg_lo, pj == pg_hi - 1);
           continue;
         }
@@ -289,17 +298,18 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
         // always in hand and the claim behind them is in flight while a page waits for its stage, which keeps the
         // counter's round trip off the critical path and tells at issue time whether a page is the segment's
         // last one: it is exactly when the claim behind it is past the end (claims only grow).
-        const int n_b = cum[b + 1] - c0s;
+        const int n_b = cb1 - c0s;
         int32_t* counter = next + static_cast<size_t>(rb) * B + b;
         int head = 0x7fffffff;
         if (lane < kStages) head = atomicAdd(counter, 1);
+        prefetch_table(b, 0, n_b);  // in flight together with the claim
         int c0 = __shfl_sync(0xffffffffu, head, 0), c1 = __shfl_sync(0xffffffffu, head, 1), c2 = __shfl_sync(0xffffffffu, head, 2);
         { int t; if (c0 > c1) { t = c0; c0 = c1; c1 = t; } if (c1 > c2) { t = c1; c1 = c2; c2 = t; } if (c0 > c1) { t = c0; c0 = c1; c1 = t; } }
         if (c0 >= n_b) {  // the others have taken everything: the combine still expects a partial from this slot
           if (rb * kRowBlock + lane < SH) partial_lse[static_cast<size_t>(part + b) * SH + rb * kRowBlock + lane] = -INFINITY;
           continue;
         }
-        issue_queries(b, part + b);
+        issue_queries(b, part + b, L);
         bool first = true;
         while (c0 < n_b) {
           int pend = 0x7fffffff;
