@@ -501,7 +501,9 @@ cudaError_t launch_combine(const transmla_params_t& p, int G, const int32_t* cum
                            int32_t* dev_status, cudaStream_t stream) {
   (void)dev_status;
   const int BS = p.batch * p.q_len;
-  const int rows = BS <= 64 ? 8 : 16;  // smaller blocks when there are few query rows, for more parallelism
+  // 8 rows per block while the register-prefetching variant runs (few query rows, more parallelism), 16 beyond:
+  // at 64 query rows that is 256 blocks, one wave at two blocks per SM, instead of 512
+  const int rows = BS <= 32 ? 8 : 16;
   const int zsplit = (BS <= 64 && p.v_dim >= 128) ? 2 : 1;
   dim3 grid(p.num_heads, (BS + rows - 1) / rows, zsplit);
   const size_t smem = 2 * kCombineRows * (p.kv_lora_rank + 8) * sizeof(__nv_bfloat16);
