@@ -199,13 +199,15 @@ typedef struct {
   const void* w_o;       /* [D, H*dv]:  y = W_O [o_1; ...; o_H]  (Eq. 9, last line) */
 } transmla_layer_weights_t;
 
-/* Bytes of device scratch transmla_layer_decode_step needs (c^Q, q^C, q^R and the attention output, bf16). */
+/* Bytes of device scratch transmla_layer_decode_step needs: c^Q, q^C, q^R and the attention output (bf16), plus
+ * the partial sums and arrival counters of the K-sliced linear maps used from 48 new tokens on. */
 size_t transmla_layer_scratch_bytes(const transmla_params_t* params /* host */, int32_t q_lora_rank);
 
 /* The whole attention layer for the S newest tokens of every sequence, x [B, S, D] -> y [B, S, D] (device bf16):
  * queries (Eq. 8 right column, RoPE of q^R at position L_b - S + s), then transmla_decode_step (append, absorb,
  * split-KV decode, combine), then the output projection W_O (Eq. 9, last line).  The linear maps are skinny
- * GEMMs with M = B*S that stream their weights once.  Needs D, H*dv (and r_q) multiples of 256; other rules
+ * GEMMs with M = B*S that stream their weights once (mma.sync tiles; from 48 tokens on the large maps run as
+ * TMA + tcgen05 tiles of 128 features with K cut into slices).  Needs D, H*dv (and r_q) multiples of 256; other rules
  * as for transmla_decode_step.  `scratch` is device memory of transmla_layer_scratch_bytes bytes, 256-byte
  * aligned. */
 transmla_status_t transmla_layer_decode_step(const transmla_params_t* params /* host */,

@@ -1,25 +1,13 @@
 // Linear maps either side of the attention (Eq. 8 right column: queries; Eq. 9 last line: W_O), as skinny GEMMs
 // y[M, N] = x[M, K] w[N, K]^T with M = the step's new tokens.  They stream their weights once; a block owns 8
 // output features (see skinny_gemm.cuh).  One launch may hold two jobs (q^C and q^R share their input).
+#include <algorithm>
+
 #include "common.cuh"
+#include "linear_args.cuh"
 #include "skinny_gemm.cuh"
 
 namespace transmla {
-
-struct LinearJob {
-  const __nv_bfloat16* x;   // [M, K]
-  const __nv_bfloat16* w;   // [N, K]
-  __nv_bfloat16* out;       // [M, N]
-  int N, K;
-  int rope_d;               // > 0: consecutive blocks of rope_d output features are rotated (Eq. 1, d := rope_d)
-};
-struct LinearArgs {
-  LinearJob job[2];
-  int n_jobs, M, S, t_splits;
-  const int32_t* pos_base;  // position of token (b, s) = pos_base[b] + pos_shift + s (used by rotated jobs only)
-  int pos_shift;
-  float theta;
-};
 
 // MAXMT x 16 tokens per pass, NT x 8 output features per block.
 template <int MAXMT, int NT>
@@ -82,6 +70,15 @@ size_t transmla_layer_scratch_bytes(const transmla_params_t* p, int32_t q_lora_r
   off = round_up(off + M * H * p->qk_nope_dim * 2, kAlign);
   off = round_up(off + M * H * p->qk_rope_dim * 2 + 16, kAlign);
   off = round_up(off + M * H * p->v_dim * 2, kAlign);
+  // tcgen05 linear maps: partial results of the K slices (largest of the three launches) and arrival counters
+  const int Mi = static_cast<int>(M), D = p->hidden_dim, Kq = q_lora_rank ? q_lora_rank : D;
+  const int tiles_dq = q_lora_rank / 128, tiles_q = static_cast<int>(H) * (p->qk_nope_dim + p->qk_rope_dim) / 128, tiles_o = D / 128;
+  size_t partial = 0;
+  if (tiles_dq > 0) partial = std::max(partial, linear_sm100_partial_bytes(tiles_dq, D, Mi));
+  if (tiles_q > 0) partial = std::max(partial, linear_sm100_partial_bytes(tiles_q, Kq, Mi));
+  if (tiles_o > 0) partial = std::max(partial, linear_sm100_partial_bytes(tiles_o, static_cast<int>(H) * p->v_dim, Mi));
+  off = round_up(off + partial, kAlign);
+  off = round_up(off + linear_sm100_counter_bytes(std::max(tiles_dq, std::max(tiles_q, tiles_o)) + 1, Mi), kAlign);
   return off;
 }
 
@@ -109,8 +106,29 @@ transmla_status_t transmla_layer_decode_step(const transmla_params_t* p, const t
   auto* cq = reinterpret_cast<__nv_bfloat16*>(base + off);      off = round_up(off + static_cast<size_t>(M) * rq * 2, kAlign);
   auto* q_nope = reinterpret_cast<__nv_bfloat16*>(base + off);  off = round_up(off + static_cast<size_t>(M) * H * p->qk_nope_dim * 2, kAlign);
   auto* q_pe = reinterpret_cast<__nv_bfloat16*>(base + off);    off = round_up(off + static_cast<size_t>(M) * H * p->qk_rope_dim * 2 + 16, kAlign);
-  auto* attn = reinterpret_cast<__nv_bfloat16*>(base + off);
+  auto* attn = reinterpret_cast<__nv_bfloat16*>(base + off);                          off = round_up(off + static_cast<size_t>(M) * H * p->v_dim * 2, kAlign);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // tcgen05 linear maps (feature counts that are multiples of 128): scratch for the K slices and their counters
+  const int tiles_dq = rq / 128, tiles_q = H * (p->qk_nope_dim + p->qk_rope_dim) / 128, tiles_o = D / 128;
+  size_t partial_bytes = 0;
+  if (tiles_dq > 0) partial_bytes = std::max(partial_bytes, linear_sm100_partial_bytes(tiles_dq, D, M));
+  if (tiles_q > 0) partial_bytes = std::max(partial_bytes, linear_sm100_partial_bytes(tiles_q, Kq, M));
+  if (tiles_o > 0) partial_bytes = std::max(partial_bytes, linear_sm100_partial_bytes(tiles_o, Ko, M));
+  auto* lin_partial = reinterpret_cast<float*>(base + off);                          off = round_up(off + partial_bytes, kAlign);
+  auto* lin_counters = reinterpret_cast<int32_t*>(base + off);
+  const size_t counter_bytes = linear_sm100_counter_bytes(std::max(tiles_dq, std::max(tiles_q, tiles_o)) + 1, M);
+  bool counters_cleared = false;
+  // One linear launch: the tcgen05 kernel where the shapes allow it, the mma.sync tiles otherwise.  The counters
+  // of the tcgen05 kernel must be zero before its first launch of this call; every launch leaves them at zero.
+  auto run_linear = [&](const LinearArgs& la) -> cudaError_t {
+    if (!linear_sm100_supported(la)) return launch_linear(la, s);
+    if (!counters_cleared) {
+      cudaError_t e = cudaMemsetAsync(lin_counters, 0, counter_bytes, s);
+      if (e != cudaSuccess) return e;
+      counters_cleared = true;
+    }
+    return launch_linear_sm100(la, lin_partial, lin_counters, dev_status, s);
+  };
   const auto* xin = static_cast<const __nv_bfloat16*>(x);
 
   LinearArgs a = {};
@@ -118,13 +136,13 @@ transmla_status_t transmla_layer_decode_step(const transmla_params_t* p, const t
   if (low_rank) {  // c^Q = W_DQ x
     a.n_jobs = 1;
     a.job[0] = {xin, static_cast<const __nv_bfloat16*>(w->w_dq), cq, rq, D, 0};
-    if (launch_linear(a, s) != cudaSuccess) return TRANSMLA_ERR_CUDA;
+    if (run_linear(a) != cudaSuccess) return TRANSMLA_ERR_CUDA;
   }
   const __nv_bfloat16* qin = low_rank ? cq : xin;
   a.n_jobs = p->qk_rope_dim > 0 ? 2 : 1;  // q^C = W_UQ c^Q and q^R = RoPE(W_QR c^Q, t) in one launch
   a.job[0] = {qin, static_cast<const __nv_bfloat16*>(w->w_uq), q_nope, H * p->qk_nope_dim, Kq, 0};
   a.job[1] = {qin, static_cast<const __nv_bfloat16*>(w->w_qr), q_pe, H * p->qk_rope_dim, Kq, p->qk_rope_dim};
-  if (launch_linear(a, s) != cudaSuccess) return TRANSMLA_ERR_CUDA;
+  if (run_linear(a) != cudaSuccess) return TRANSMLA_ERR_CUDA;
 
   transmla_status_t st = transmla_decode_step(p, x, q_nope, q_pe, page_table, seqlens, w->w_dkv_kr, w->w_uk, w->w_uv, cache,
                                               workspace, workspace_bytes, attn, nullptr, dev_status, stream);
@@ -132,7 +150,7 @@ transmla_status_t transmla_layer_decode_step(const transmla_params_t* p, const t
 
   a.n_jobs = 1;  // y = W_O [o_1; ...; o_h]
   a.job[0] = {attn, static_cast<const __nv_bfloat16*>(w->w_o), static_cast<__nv_bfloat16*>(y), D, Ko, 0};
-  if (launch_linear(a, s) != cudaSuccess) return TRANSMLA_ERR_CUDA;
+  if (run_linear(a) != cudaSuccess) return TRANSMLA_ERR_CUDA;
   return TRANSMLA_OK;
 }
 

@@ -290,7 +290,11 @@ def test_decode_step_from_host_buffers(pinned):
 # ------------------------------------------------------------------ whole layer: queries, attention, W_O
 @pytest.mark.parametrize('shape,seqlens,rq', [(synth.TINY, [17, 64, 130], 0), (synth.TINY, [5, 70], 256),
                                                (synth.LLAMA2_7B, [300, 65, 1024], 0), (synth.LLAMA2_7B, [200, 64], 512),
-                                               (synth.QWEN25_72B, [131, 700], 0)])
+                                               (synth.QWEN25_72B, [131, 700], 0),
+                                               # 48 and more new tokens: the large maps run on the tcgen05 kernel
+                                               (synth.LLAMA2_7B, [70 + 3 * i for i in range(50)], 0),
+                                               (synth.LLAMA2_7B, [64 + i for i in range(130)], 512),
+                                               (synth.QWEN25_72B, [66 + 5 * i for i in range(25)], 0)])
 def test_layer_decode_step(shape, seqlens, rq):
     B, S = len(seqlens), shape.S
     scale = gu.mla_scale(shape)
