@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the absorbed-MLA decode step (append + absorb + split-KV decode + combine).
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME] [--layer]
 
 One step = one pass of the whole path over one batch: every sequence appends its new token's
 latent and decodes over its cached tokens.  The default workload is the LLaMA-2-7B-converted
@@ -260,6 +260,37 @@ def run_ours(args, name, shape, seqlens, seed):
     h2d = sum(v.numel() * v.element_size() for v in h.values())
     d2h = h_out.numel() * 2 + h_lse.numel() * 4 + 4
 
+    layer = None
+    if args.layer:
+        # the whole attention layer (queries -> the step above -> W_O) on device buffers; its weights rotate too
+        lws = []
+        for i in range(args.layer_weight_copies):
+            lw = synth.make_layer_weights(shape, seed + 10 + i, q_lora_rank=args.q_lora_rank, device='cuda')
+            lw.update(w_dkv_kr=weights[i % n_w][0], w_uk=weights[i % n_w][1], w_uv=weights[i % n_w][2])
+            lws.append(lw)
+        scratch = torch.empty(binding.transmla_layer_scratch_bytes(params, args.q_lora_rank), dtype=torch.uint8, device='cuda')
+        y = torch.empty(B, S, shape.D, dtype=torch.bfloat16, device='cuda')
+
+        def layer_step(i):
+            binding.transmla_layer_decode_step(params, lws[i % len(lws)], ac['x'], dc['page_table'], dc['seqlens'],
+                                               caches[i % n_copies], ws, scratch, y, status, stream)
+        for i in range(max(args.warmup, 3)):
+            layer_step(i)
+        barrier()
+        l0, l1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        l0.record(stream)
+        for i in range(args.steps):
+            layer_step(i)
+        l1.record(stream)
+        barrier()
+        word = int(status.item())
+        assert word == 0, f'device status word {word:#x} after the layer steps'
+        layer_ms = replicas.max_over_ranks([l0.elapsed_time(l1)], device='cuda')[0] / args.steps
+        lbytes = sum(t.numel() * t.element_size() for t in lws[0].values())
+        layer = {'ms_per_step': layer_ms, 'tokens_per_s': B * S * world / (layer_ms * 1e-3), 'weight_bytes': lbytes,
+                 'q_lora_rank': args.q_lora_rank, 'launches_per_step': 6 + (1 if args.q_lora_rank else 0),
+                 'gbs_weights_plus_cache': (lbytes + sum(seqlens) * shape.row * 2) / (layer_ms * 1e-3) / 1e9}
+
     ms_total, e2e_ms = replicas.max_over_ranks([ms_total, e2e_s * 1e3], device='cuda')
     if rank != 0:
         if world > 1:
@@ -275,7 +306,7 @@ def run_ours(args, name, shape, seqlens, seed):
     peak, peak_kind = measured_hbm_peak()
     # ncu dram__bytes_read.sum + dram__bytes_write.sum of one split-KV launch on the default workload
     # (profiles/decode_sm100_llama2-7b_b16_8k.md); other workloads have no capture
-    traffic = 155.60e6 if name == 'llama2-7b-mla_b16_8k' and world == 1 else None
+    traffic = 156.93e6 if name == 'llama2-7b-mla_b16_8k' and world == 1 else None
     line = {
         'metric': METRIC, 'value': replicas.whole_job_rate(B * S, args.steps, ms_total), 'unit': 'tokens/s', 'n_gpus': world,
         'steps': args.steps, 'warmup': max(args.warmup, 3), 'ms_per_step': ms_step, 'higher_is_better': True,
@@ -297,6 +328,8 @@ def run_ours(args, name, shape, seqlens, seed):
         'gpu_launches': KERNELS_PER_STEP * args.steps,
         'clocks': clocks,
     }
+    if layer is not None:
+        line['layer'] = layer
     if world == 1 and not args.no_cpu_baseline:
         line['cpu_baseline'] = cpu_baseline(shape, seqlens, seed, scale)
     print(json.dumps(line))
@@ -314,6 +347,9 @@ def main():
     ap.add_argument('--cache-copies', type=int, default=4)
     ap.add_argument('--weight-copies', type=int, default=12)
     ap.add_argument('--no-cpu-baseline', action='store_true')
+    ap.add_argument('--layer', action='store_true', help='also time the whole layer step (queries, attention, W_O)')
+    ap.add_argument('--q-lora-rank', type=int, default=0, help='low-rank queries for --layer (0: full rank)')
+    ap.add_argument('--layer-weight-copies', type=int, default=6)
     args = ap.parse_args()
     w = workloads()
     if args.workload not in w:
