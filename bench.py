@@ -47,6 +47,15 @@ def measured_hbm_peak():
         return 6650.0, 'fallback'
 
 
+def measured_tensor_peak():
+    """Dense bf16 TFLOP/s of a GEMM timed alone (the split-KV kernel is timed alone too)."""
+    path = os.path.join(ROOT, 'MEASURED_PEAKS.json')
+    try:
+        return float(json.load(open(path))['bf16_tflops']), 'measured'
+    except Exception:
+        return 1590.0, 'fallback'
+
+
 class ClockSampler:
     """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
     FIELDS = ('clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,'
@@ -304,6 +313,10 @@ def run_ours(args, name, shape, seqlens, seed):
     algo_bytes = cache_bytes + q_hat_bytes                           # per split-KV launch
     achieved = algo_bytes / (kernel_ms * 1e-3) / 1e9
     peak, peak_kind = measured_hbm_peak()
+    # the other roof: 2 * (r + dR) flop for a score and 2 * r for its share of the weighted sum, per query row and token
+    flops = 2.0 * (shape.row + shape.r) * H * S * sum(seqlens)
+    tpeak, tpeak_kind = measured_tensor_peak()
+    tflops = flops / (kernel_ms * 1e-3) / 1e12
     # ncu dram__bytes_read.sum + dram__bytes_write.sum of one split-KV launch on the default workload
     # (profiles/decode_sm100_llama2-7b_b16_8k.md); other workloads have no capture
     traffic = 156.93e6 if name == 'llama2-7b-mla_b16_8k' and world == 1 else None
@@ -322,7 +335,9 @@ def run_ours(args, name, shape, seqlens, seed):
         'decode_kernel_us': kernel_ms * 1e3, 'decode_kernel_launches_timed': len(kev),
         'roofline': {'bound': 'hbm', 'achieved': achieved, 'peak': peak, 'unit': 'GB/s', 'frac': achieved / peak,
                      'peak_kind': f'{peak_kind} copy bandwidth', 'frac_of_8tbs': achieved / NOMINAL_HBM_GBS,
-                     'kernel': 'split-KV decode', 'algorithmic_bytes_per_launch': algo_bytes, 'traffic': traffic},
+                     'kernel': 'split-KV decode', 'algorithmic_bytes_per_launch': algo_bytes, 'traffic': traffic,
+                     'tensor': {'achieved_tflops': tflops, 'peak_tflops': tpeak, 'peak_kind': f'{tpeak_kind} bf16 GEMM',
+                                'frac': tflops / tpeak, 'flops_per_launch': flops}},
         'e2e': {'value': replicas.whole_job_rate(B * S, args.steps, e2e_ms), 'unit': 'tokens/s',
                 'h2d_bytes_per_step': h2d, 'd2h_bytes_per_step': d2h, 'ms_per_step': e2e_ms / args.steps},
         'gpu_launches': KERNELS_PER_STEP * args.steps,
@@ -340,8 +355,8 @@ def run_ours(args, name, shape, seqlens, seed):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument('--gpus', type=int, default=1)
-    ap.add_argument('--steps', type=int, default=200)
-    ap.add_argument('--warmup', type=int, default=10)
+    ap.add_argument('--steps', type=int, default=1000)
+    ap.add_argument('--warmup', type=int, default=20)
     ap.add_argument('--impl', default='ours', choices=['ours', 'reference'])
     ap.add_argument('--workload', default='llama2-7b-mla_b16_8k')
     ap.add_argument('--cache-copies', type=int, default=4)
