@@ -321,15 +321,16 @@ def test_layer_decode_step(shape, seqlens, rq):
 
 
 # ------------------------------------------------------------------ pages claimed at run time (G = 0, many CTAs per sequence)
-@pytest.mark.parametrize('seqlens', [[4096 + 17, 2100], [8192], [64 * 40, 64 * 41 + 1, 3000]])
-def test_dynamic_page_claims_match_the_oracle(seqlens):
+@pytest.mark.parametrize('shape,seqlens', [(synth.LLAMA2_7B, [4096 + 17, 2100]), (synth.LLAMA2_7B, [8192]),
+                                           (synth.LLAMA2_7B, [64 * 40, 64 * 41 + 1, 3000]),
+                                           (synth.QWEN25_72B, [4000]), (synth.QWEN25_72B, [3001, 2990])])
+def test_dynamic_page_claims_match_the_oracle(shape, seqlens):
     # With G = 0 and at least 8 partitions per sequence the CTAs of a sequence take its pages from a counter, so
     # the grouping of pages into partials depends on timing: what is unique is the combined result.
-    shape = synth.LLAMA2_7B
     scale = gu.mla_scale(shape)
     case = synth.make_decode_case(shape, seqlens, seed=23, nan_tails=True)
     dev = gu.to_dev(case)
-    only = [(b, 0, h) for b in range(len(seqlens)) for h in (0, 5, 31)]
+    only = [(b, s, h) for b in range(len(seqlens)) for s in range(shape.S) for h in (0, 5, shape.H - 1)]
     want, want_lse = gu.oracle_decode(shape, case, scale, only=only)
     idx = tuple(np.array(only).T)
     for _ in range(3):
