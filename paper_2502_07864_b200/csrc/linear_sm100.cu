@@ -8,9 +8,13 @@
 // tokens (16 <= T <= 256, tokens padded to a multiple of 16; rows beyond M read as zero through the tensor map).
 // Per CTA the shared-memory traffic is (128 + T) x K_slice x 2 bytes, i.e. the activations are re-read once per
 // 128 features, not once per 8 or 32 as in the mma.sync tiles of skinny_gemm.cuh.
-// K is cut into `splits` slices so that every SM streams weights (N / 128 tiles alone would occupy 32-48 SMs);
-// each slice's partial goes to a scratch buffer, and the CTA that arrives last at the tile's counter adds the
-// slices in a fixed order, applies RoPE where asked and writes bf16 (no float atomics: reruns give the same bits).
+// K is cut into `splits` slices so that every SM streams weights (N / 128 tiles alone would occupy 32-48 SMs).
+// The slices of a tile are the CTAs of one thread-block cluster: each leaves its fp32 partial in its own shared
+// memory (the ring is free by then), and after a cluster barrier every CTA adds the slices of its share of the
+// tokens in slice order, reading the others' shared memory directly, applies RoPE where asked and writes bf16 (no
+// float atomics: reruns give the same bits).  If the clusters do not all fit on the device at once, or there are
+// more than 8 slices, the partials go through a scratch buffer instead and the CTA that arrives last at the tile's
+// counter adds them.
 //
 // Warps: 0 TMA producer, 1 MMA issuer, 2-5 epilogue (each owns the 32 tensor-memory lanes of its quadrant).
 #include "common.cuh"
@@ -30,18 +34,83 @@ constexpr int kLinThreads = 192;
 constexpr int kLinSmemBytes = kLinRingBytes + 256 + 1024;
 enum { LB_FULL = 0, LB_EMPTY = kLinMaxStages, LB_DONE = 2 * kLinMaxStages };
 
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// fp32 at the same shared-memory offset in the CTA of rank `rank` of this cluster
+__device__ __forceinline__ float ld_cluster_f32(const float* local, uint32_t rank) {
+  uint32_t remote;
+  float v;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(local)), "r"(rank));
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
+  return v;
+}
+
 struct LinSm100Params {
   __nv_bfloat16* out[2];   // [M, N_j]
   int N[2];                // output features of job j (multiples of 128)
   int rope_d[2];           // > 0: consecutive blocks of rope_d features are rotated (Eq. 1, d := rope_d)
   int n_jobs, M, S, K, splits;
   int stages;              // ring depth: as many (weight tile + activation box) stages as fit
+  int cluster;             // 1: the slices of a tile are the CTAs of one cluster and meet through distributed shared memory
   int x_box_rows;          // rows of the activation box (tokens of a full block, padded to 16); also the row stride of `partial`
   const int32_t* pos_base; // position of token (b, s) = pos_base[b] + pos_shift + s (rotated jobs only)
   int pos_shift;
   float theta;
   float* partial;          // [token block][tile][split][T][128] fp32 (splits > 1)
   int32_t* counters;       // [token block][tile], zero before the launch; left at zero
+};
+
+// RoPE of Eq. 1 in the epilogue, rounding and the store.  The even lane of a pair holds the real part, the odd one
+// the imaginary part.  Angle = position x theta^(-2l/d), reduced to [-pi, pi] before sine and cosine.  The
+// reduction runs in fp32 with the frequency as a (hi, lo) pair and 2*pi as three constants whose products with the
+// turn count are formed exactly inside the fused multiply-adds (positions up to 2^20 keep an angle error below
+// 1e-5 rad); the double-precision units of this chip are too slow to do it for every (token, pair).  Tokens are
+// taken two at a time: the even lane works out the angle of the first, the odd lane that of the second, and they
+// swap.
+struct LinRope {
+  float f_hi = 0.f, f_lo = 0.f;
+  int rope_d, S, pos_shift;
+  const int32_t* pos_base;
+  __device__ LinRope(const LinSm100Params& p, int feature, int rope_d_)
+      : rope_d(rope_d_), S(p.S), pos_shift(p.pos_shift), pos_base(p.pos_base) {
+    if (rope_d > 0) {
+      const double inv_freq = exp2(-2.0 * ((feature % rope_d) >> 1) / rope_d * log2(static_cast<double>(p.theta)));
+      f_hi = static_cast<float>(inv_freq);
+      f_lo = static_cast<float>(inv_freq - static_cast<double>(f_hi));
+    }
+  }
+  __device__ void sincos_at(int tok, float& sn, float& cs) const {
+    const float pos = static_cast<float>(pos_base[tok / S] + pos_shift + tok % S);
+    const float a = pos * f_hi;
+    const float e = fmaf(pos, f_hi, -a) + pos * f_lo;          // what the rounded product left out
+    const float k = rintf(a * 0.15915494309189535f);          // whole turns
+    float r = fmaf(-k, 6.28125f, a);                           // 2*pi = 6.28125 + 0.001934051513671875 + 1.2556659146e-6
+    r = fmaf(-k, 0.001934051513671875f, r);
+    r = fmaf(-k, 1.2556659146e-6f, r) + e;
+    sincosf(r, &sn, &cs);
+  }
+  // values of `feature` for tokens t0 + t and t0 + t + 1 (the second only if has_b): rotate, round, store.
+  // Called by all 32 lanes of a warp together.
+  __device__ void finish2(__nv_bfloat16* out, int N, int feature, int t0, int t, float va, float vb, bool has_b, int lane) const {
+    const float oa = __shfl_xor_sync(0xffffffffu, va, 1), ob = __shfl_xor_sync(0xffffffffu, vb, 1);
+    const bool odd = (lane & 1) != 0;
+    float re_a = odd ? oa : va, im_a = odd ? va : oa, re_b = odd ? ob : vb, im_b = odd ? vb : ob;
+    if (rope_d > 0) {
+      float sn = 0.f, cs = 1.f;
+      sincos_at(t0 + t + ((odd && has_b) ? 1 : 0), sn, cs);    // even lane: first token; odd lane: second
+      const float sn_o = __shfl_xor_sync(0xffffffffu, sn, 1), cs_o = __shfl_xor_sync(0xffffffffu, cs, 1);
+      const float sn_a = odd ? sn_o : sn, cs_a = odd ? cs_o : cs;
+      const float sn_b = (odd || !has_b) ? sn : sn_o, cs_b = (odd || !has_b) ? cs : cs_o;
+      const float ra = re_a * cs_a - im_a * sn_a, ia = im_a * cs_a + re_a * sn_a;
+      const float rb = re_b * cs_b - im_b * sn_b, ib = im_b * cs_b + re_b * sn_b;
+      re_a = ra; im_a = ia; re_b = rb; im_b = ib;
+    }
+    if (!odd) {
+      *reinterpret_cast<uint32_t*>(out + static_cast<size_t>(t0 + t) * N + feature) = pack_bf16(re_a, im_a);
+      if (has_b) *reinterpret_cast<uint32_t*>(out + static_cast<size_t>(t0 + t + 1) * N + feature) = pack_bf16(re_b, im_b);
+    }
+  }
 };
 
 __global__ void __launch_bounds__(kLinThreads, 1)
@@ -151,48 +220,8 @@ linear_sm100_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_con
     pdl_wait();  // the scratch buffer, the counters and the output may still be in use by earlier kernels
     mbar_wait(bar(LB_DONE), 0, abort_flag, dev_status);
     tc_fence_after();
-    // RoPE of Eq. 1 in the epilogue.  The even lane of a pair holds the real part, the odd one the imaginary part.
-    // Angle = position x theta^(-2l/d), reduced to [-pi, pi] before sine and cosine.  The reduction runs in fp32
-    // with the frequency as a (hi, lo) pair and 2*pi as three constants whose products with the turn count are
-    // formed exactly inside the fused multiply-adds (positions up to 2^20 keep an angle error below 1e-5 rad); the
-    // double-precision units of this chip are too slow to do it for every (token, pair).  Tokens are taken two
-    // at a time: the even lane works out the angle of the first, the odd lane that of the second, and they swap.
-    float f_hi = 0.f, f_lo = 0.f;
-    if (rope_d > 0) {
-      const double inv_freq = exp2(-2.0 * (((f0 + fl) % rope_d) >> 1) / rope_d * log2(static_cast<double>(p.theta)));
-      f_hi = static_cast<float>(inv_freq);
-      f_lo = static_cast<float>(inv_freq - static_cast<double>(f_hi));
-    }
-    auto sincos_at = [&](int tok, float& sn, float& cs) {
-      const float pos = static_cast<float>(p.pos_base[tok / p.S] + p.pos_shift + tok % p.S);
-      const float a = pos * f_hi;
-      const float e = fmaf(pos, f_hi, -a) + pos * f_lo;          // what the rounded product left out
-      const float k = rintf(a * 0.15915494309189535f);          // whole turns
-      float r = fmaf(-k, 6.28125f, a);                           // 2*pi = 6.28125 + 0.001934051513671875 + 1.2556659146e-6
-      r = fmaf(-k, 0.001934051513671875f, r);
-      r = fmaf(-k, 1.2556659146e-6f, r) + e;
-      sincosf(r, &sn, &cs);
-    };
-    // values of feature f0 + fl for tokens t0 + t and t0 + t + 1 (the second only if has_b): rotate, round, store
-    auto finish2 = [&](int t, float va, float vb, bool has_b) {
-      const float oa = __shfl_xor_sync(0xffffffffu, va, 1), ob = __shfl_xor_sync(0xffffffffu, vb, 1);
-      const bool odd = (lane & 1) != 0;
-      float re_a = odd ? oa : va, im_a = odd ? va : oa, re_b = odd ? ob : vb, im_b = odd ? vb : ob;
-      if (rope_d > 0) {
-        float sn = 0.f, cs = 1.f;
-        sincos_at(t0 + t + ((odd && has_b) ? 1 : 0), sn, cs);    // even lane: first token; odd lane: second
-        const float sn_o = __shfl_xor_sync(0xffffffffu, sn, 1), cs_o = __shfl_xor_sync(0xffffffffu, cs, 1);
-        const float sn_a = odd ? sn_o : sn, cs_a = odd ? cs_o : cs;
-        const float sn_b = (odd || !has_b) ? sn : sn_o, cs_b = (odd || !has_b) ? cs : cs_o;
-        const float ra = re_a * cs_a - im_a * sn_a, ia = im_a * cs_a + re_a * sn_a;
-        const float rb = re_b * cs_b - im_b * sn_b, ib = im_b * cs_b + re_b * sn_b;
-        re_a = ra; im_a = ia; re_b = rb; im_b = ib;
-      }
-      if (!odd) {
-        *reinterpret_cast<uint32_t*>(out + static_cast<size_t>(t0 + t) * N + f0 + fl) = pack_bf16(re_a, im_a);
-        if (has_b) *reinterpret_cast<uint32_t*>(out + static_cast<size_t>(t0 + t + 1) * N + f0 + fl) = pack_bf16(re_b, im_b);
-      }
-    };
+    LinRope rope(p, f0 + fl, rope_d);
+    auto finish2 = [&](int t, float va, float vb, bool has_b) { rope.finish2(out, N, f0 + fl, t0, t, va, vb, has_b, lane); };
     const size_t tile_id = static_cast<size_t>(blockIdx.y) * tiles + tile;
     const size_t slice_elems = static_cast<size_t>(p.x_box_rows) * kLinBM;
     float* my_partial = p.partial + (tile_id * p.splits + split) * slice_elems;
@@ -206,6 +235,10 @@ linear_sm100_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_con
           const bool has_b = c + j + 1 < T;
           if (p.splits == 1) {
             finish2(c + j, __uint_as_float(v[j]), __uint_as_float(v[j + 1]), has_b);
+          } else if (p.cluster) {  // the ring is free: every MMA of this CTA has retired
+            float* part_s = reinterpret_cast<float*>(sm);
+            part_s[(c + j) * kLinBM + fl] = __uint_as_float(v[j]);
+            if (has_b) part_s[(c + j + 1) * kLinBM + fl] = __uint_as_float(v[j + 1]);
           } else {
             my_partial[static_cast<size_t>(c + j) * kLinBM + fl] = __uint_as_float(v[j]);
             if (has_b) my_partial[static_cast<size_t>(c + j + 1) * kLinBM + fl] = __uint_as_float(v[j + 1]);
@@ -213,7 +246,7 @@ linear_sm100_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_con
         }
       }
     }
-    if (p.splits > 1) {
+    if (p.splits > 1 && !p.cluster) {
       // the slice that arrives last at the tile's counter adds all slices, in slice order
       __threadfence();
       asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -245,6 +278,37 @@ linear_sm100_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_con
       }
     }
     tc_fence_before();
+  }
+
+  if (p.cluster && p.splits > 1) {
+    // ---- the slices of the tile meet: every CTA of the cluster has its partial [T][128] in its own shared memory;
+    // CTA `split` adds the slices of its share of the tokens in slice order, reading the others' memory directly
+    cluster_sync_all();
+    if (warp >= 2) {
+      const int quad = warp & 3, fl = quad * 32 + lane;
+      const int N = p.N[job], rope_d = p.rope_d[job];
+      __nv_bfloat16* out = p.out[job];
+      const float* part_s = reinterpret_cast<const float*>(sm);
+      const int share = (((T + p.splits - 1) / p.splits) + 1) & ~1;  // even, so that token pairs stay together
+      const int ts = split * share, te = min(T, ts + share);
+      LinRope rope(p, f0 + fl, rope_d);
+      for (int tb = ts; tb < te; tb += 8) {
+        float acc[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) acc[u] = 0.f;
+        for (int s = 0; s < p.splits; ++s) {
+          float v[8];
+#pragma unroll
+          for (int u = 0; u < 8; ++u) v[u] = tb + u < te ? ld_cluster_f32(part_s + (tb + u) * kLinBM + fl, s) : 0.f;
+#pragma unroll
+          for (int u = 0; u < 8; ++u) acc[u] += v[u];
+        }
+#pragma unroll
+        for (int u = 0; u < 8; u += 2)
+          if (tb + u < te) rope.finish2(out, N, f0 + fl, t0, tb + u, acc[u], acc[u + 1], tb + u + 1 < te, lane);
+      }
+    }
+    cluster_sync_all();  // nobody leaves while its memory may still be read
   }
 
   // ---- teardown
@@ -279,11 +343,12 @@ int linear_sm100_splits(int n_tiles, int K) {
   return s < 1 ? 1 : s;
 }
 
-// Where this kernel is used.  Its CTAs take the whole shared memory (they cannot start while blocks of the kernel
-// before them are still resident) and meet through a scratch buffer at the end, which costs about 6 us per launch
-// whatever the size; the mma.sync tiles of linear.cu have neither cost but re-read the activations once per 32
-// features.  Measured on the LLaMA-2-7B shape the tcgen05 kernel wins from about 48 tokens on, with long rows of
-// weights (K >= 2048) and at least 24 tiles of 128 features (B = 128: 108 -> 92 us for the layer's two large maps).
+// Where this kernel is used.  Its CTAs take the whole shared memory, so they cannot start while blocks of the kernel
+// before them are still resident, and the slices of a tile have to meet at the end; the mma.sync tiles of linear.cu
+// have neither cost but re-read the activations once per 32 features.  Measured on the LLaMA-2-7B shape (layer
+// step, pipelined) the tcgen05 kernel wins from about 48 tokens on, with long rows of weights (K >= 2048) and at
+// least 24 tiles of 128 features: B = 128: 108 -> 82 us for the layer's two large maps; at 16 tokens it is level
+// with the mma.sync tiles and at 1 token 13 us slower.
 bool linear_sm100_supported(const LinearArgs& a) {
   if (a.n_jobs < 1 || a.n_jobs > 2 || a.M < 48 || a.job[0].K < 2048) return false;
   int tiles = 0;
@@ -336,8 +401,34 @@ cudaError_t launch_linear_sm100(const LinearArgs& a, float* partial, int32_t* co
     attr_set = true;
   }
   dim3 grid(tiles * p.splits, (a.M + kLinMaxT - 1) / kLinMaxT);
-  return launch_pdl(linear_sm100_kernel, grid, dim3(kLinThreads), static_cast<size_t>(kLinSmemBytes), stream, wmap[0], wmap[1],
-                    xmap, p, dev_status);
+  // The K slices of a tile are launched as one thread-block cluster (they are neighbours in blockIdx.x) when all
+  // clusters fit on the device at once; then they meet through distributed shared memory and need neither the
+  // scratch buffer nor the counters.
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(kLinThreads);
+  cfg.dynamicSmemBytes = kLinSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  p.cluster = 0;
+  if (p.splits > 1 && p.splits <= 8) {
+    static int max_clusters[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};  // co-resident clusters of each size, asked once
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = p.splits; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+    cfg.numAttrs = 2;
+    if (max_clusters[p.splits] == 0) {
+      int n = 0;
+      if (cudaOccupancyMaxActiveClusters(&n, linear_sm100_kernel, &cfg) != cudaSuccess) { cudaGetLastError(); n = -1; }
+      max_clusters[p.splits] = n > 0 ? n : -1;
+    }
+    if (max_clusters[p.splits] >= static_cast<int>(grid.x * grid.y) / p.splits) p.cluster = 1;
+    else cfg.numAttrs = 1;
+  }
+  return cudaLaunchKernelEx(&cfg, linear_sm100_kernel, wmap[0], wmap[1], xmap, p, dev_status);
 }
 
 }  // namespace transmla
