@@ -347,7 +347,7 @@ int linear_sm100_splits(int n_tiles, int K) {
 // before them are still resident, and the slices of a tile have to meet at the end; the mma.sync tiles of linear.cu
 // have neither cost but re-read the activations once per 32 features.  Measured on the LLaMA-2-7B shape (layer
 // step, pipelined) the tcgen05 kernel wins from about 48 tokens on, with long rows of weights (K >= 2048) and at
-// least 24 tiles of 128 features: B = 128: 108 -> 82 us for the layer's two large maps; at 16 tokens it is level
+// least 24 tiles of 128 features: B = 128: 108 -> 70 us for the layer's two large maps; at 16 tokens it is level
 // with the mma.sync tiles and at 1 token 13 us slower.
 bool linear_sm100_supported(const LinearArgs& a) {
   if (a.n_jobs < 1 || a.n_jobs > 2 || a.M < 48 || a.job[0].K < 2048) return false;
@@ -400,33 +400,37 @@ cudaError_t launch_linear_sm100(const LinearArgs& a, float* partial, int32_t* co
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  dim3 grid(tiles * p.splits, (a.M + kLinMaxT - 1) / kLinMaxT);
-  // The K slices of a tile are launched as one thread-block cluster (they are neighbours in blockIdx.x) when all
-  // clusters fit on the device at once; then they meet through distributed shared memory and need neither the
-  // scratch buffer nor the counters.
+  const int token_blocks = (a.M + kLinMaxT - 1) / kLinMaxT;
+  // The K slices of a tile are launched as one thread-block cluster (they are neighbours in blockIdx.x); they then
+  // meet through distributed shared memory and need neither the scratch buffer nor the counters.  All clusters have
+  // to fit on the device at once (a cluster lives inside one GPC, so fewer fit than SMs / size suggests): the
+  // slice count is lowered until they do; if no size from 2 to 8 fits, the wanted count runs through the scratch.
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = grid;
   cfg.blockDim = dim3(kLinThreads);
   cfg.dynamicSmemBytes = kLinSmemBytes;
   cfg.stream = stream;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
   p.cluster = 0;
-  if (p.splits > 1 && p.splits <= 8) {
-    static int max_clusters[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};  // co-resident clusters of each size, asked once
-    attr[1].id = cudaLaunchAttributeClusterDimension;
-    attr[1].val.clusterDim.x = p.splits; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+  static int max_clusters[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};  // co-resident clusters of each size, asked once
+  for (int s = p.splits < 8 ? p.splits : 8; s >= 2 && !p.cluster; --s) {
+    attr[1].val.clusterDim.x = s;
+    cfg.gridDim = dim3(tiles * s, token_blocks);
     cfg.numAttrs = 2;
-    if (max_clusters[p.splits] == 0) {
+    if (max_clusters[s] == 0) {
       int n = 0;
       if (cudaOccupancyMaxActiveClusters(&n, linear_sm100_kernel, &cfg) != cudaSuccess) { cudaGetLastError(); n = -1; }
-      max_clusters[p.splits] = n > 0 ? n : -1;
+      max_clusters[s] = n > 0 ? n : -1;
     }
-    if (max_clusters[p.splits] >= static_cast<int>(grid.x * grid.y) / p.splits) p.cluster = 1;
-    else cfg.numAttrs = 1;
+    if (max_clusters[s] >= tiles * token_blocks) { p.cluster = 1; p.splits = s; }
+  }
+  if (!p.cluster) {
+    cfg.gridDim = dim3(tiles * p.splits, token_blocks);
+    cfg.numAttrs = 1;
   }
   return cudaLaunchKernelEx(&cfg, linear_sm100_kernel, wmap[0], wmap[1], xmap, p, dev_status);
 }
