@@ -192,16 +192,17 @@ static size_t absorb_smem(int dn) {
 // split the hidden dimension and meet in shared memory.  Tokens are the M dimension of the tiles.
 // Token (b, s) sits at position pos_base[b] + pos_shift + s.
 // ------------------------------------------------------------------------------------------------
+template <int MAXMT, int NT>
 __device__ void append_block(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w,
                              const int32_t* __restrict__ pos_base, int pos_shift,
                              const int32_t* __restrict__ page_table, __nv_bfloat16* __restrict__ cache,
                              int32_t* dev_status, int B, int S, int D, int r, int dR, int num_pages, int max_pages,
                              float theta, int nb, int t_splits, unsigned char* smem_raw) {
   // block nb = (token split, feature tile): with many tokens the token range is cut so that more SMs take part
-  const int K = r + dR, f_tiles = K / 8, f0 = (nb % f_tiles) * 8;
+  const int K = r + dR, f_tiles = K / (8 * NT), f0 = (nb % f_tiles) * 8 * NT;
   const int t_chunk = (((B * S + t_splits - 1) / t_splits) + 15) & ~15;
   const int t_begin = (nb / f_tiles) * t_chunk, t_end = min(B * S, t_begin + t_chunk);
-  skinny_gemm_tile(x, w, D, f0, t_begin, t_end, smem_raw, [&](int t, int pr, float re, float im) {
+  skinny_gemm_tile<MAXMT, NT>(x, w, D, f0, t_begin, t_end, smem_raw, [&](int t, int pr, float re, float im) {
     const int b = t / S, s = t % S;
     const int pos = pos_base[b] + pos_shift + s;
     const int pj = pos / kPage;
@@ -223,11 +224,15 @@ __global__ void __launch_bounds__(256) append_kernel(const __nv_bfloat16* __rest
                                                      const int32_t* __restrict__ page_table,
                                                      __nv_bfloat16* __restrict__ cache, int32_t* dev_status, int B,
                                                      int S, int D, int r, int dR, int num_pages, int max_pages,
-                                                     float theta, int t_splits) {
+                                                     float theta, int t_splits, int wide) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   pdl_trigger();
-  append_block(x, w, positions, 0, page_table, cache, dev_status, B, S, D, r, dR, num_pages, max_pages, theta,
-               blockIdx.x, t_splits, smem_raw);
+  if (wide)
+    append_block<1, 4>(x, w, positions, 0, page_table, cache, dev_status, B, S, D, r, dR, num_pages, max_pages, theta,
+                       blockIdx.x, t_splits, smem_raw);
+  else
+    append_block<kAppendMaxMT, 1>(x, w, positions, 0, page_table, cache, dev_status, B, S, D, r, dR, num_pages, max_pages,
+                                  theta, blockIdx.x, t_splits, smem_raw);
 }
 
 // Absorb blocks followed by one plan block: everything transmla_mla_decode needs before the split-KV kernel.
@@ -256,18 +261,22 @@ __global__ void __launch_bounds__(256) prologue_kernel(
     const int32_t* __restrict__ page_table, __nv_bfloat16* __restrict__ cache, const __nv_bfloat16* __restrict__ q_nope,
     const __nv_bfloat16* __restrict__ q_pe, const __nv_bfloat16* __restrict__ w_uk, __nv_bfloat16* __restrict__ q_hat,
     const int32_t* __restrict__ seqlens, int32_t* cum, int32_t* plan, int32_t* dev_status, int B, int S, int H, int D,
-    int dn, int dR, int r, int num_pages, int max_pages, float theta, int G, int t_splits) {
+    int dn, int dR, int r, int num_pages, int max_pages, float theta, int G, int t_splits, int wide) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   pdl_trigger();
   TRK_BEGIN(0);
-  const int n_append = (r + dR) / 8 * t_splits;
+  const int n_append = (r + dR) / (wide ? 32 : 8) * t_splits;
   const int r_tiles = (r + 127) / 128;
   const int bid = static_cast<int>(blockIdx.x) - 1;
   if (bid < 0) {
     plan_block(seqlens, B, G, (S * H + kRowBlock - 1) / kRowBlock, cum, plan, smem_raw);
   } else if (bid < n_append) {
-    append_block(x, w_dkv_kr, seqlens, -S, page_table, cache, dev_status, B, S, D, r, dR, num_pages, max_pages, theta,
-                 bid, t_splits, smem_raw);
+    if (wide)
+      append_block<1, 4>(x, w_dkv_kr, seqlens, -S, page_table, cache, dev_status, B, S, D, r, dR, num_pages, max_pages,
+                         theta, bid, t_splits, smem_raw);
+    else
+      append_block<kAppendMaxMT, 1>(x, w_dkv_kr, seqlens, -S, page_table, cache, dev_status, B, S, D, r, dR, num_pages,
+                                    max_pages, theta, bid, t_splits, smem_raw);
   } else {
     const int a = bid - n_append;
     absorb_block(q_nope, q_pe, w_uk, q_hat, B * S, H, dn, dR, r, a / r_tiles, a % r_tiles, smem_raw);
@@ -278,8 +287,14 @@ __global__ void __launch_bounds__(256) prologue_kernel(
 constexpr int kPrologueMaxSmem = 144 * 1024;
 
 // Token splits of the append: one per 64 new tokens, at most 4.
+// With many new tokens a block takes 32 output features and 16 tokens (activations re-read a quarter as often
+// per feature, weights four times as often per token: 384 KB per block instead of 576 KB at 128 tokens).
+static bool append_wide(const transmla_params_t& p) {
+  return p.batch * p.q_len > 32 && (p.kv_lora_rank + p.qk_rope_dim) % 32 == 0 && p.kv_lora_rank % 2 == 0;
+}
 static int append_token_splits(const transmla_params_t& p) {
   const int T = p.batch * p.q_len;
+  if (append_wide(p)) return (T + 15) / 16 > 32 ? 32 : (T + 15) / 16;
   return T <= 64 ? 1 : (T + 63) / 64 > 4 ? 4 : (T + 63) / 64;
 }
 
@@ -288,9 +303,10 @@ cudaError_t launch_append(const transmla_params_t& p, const __nv_bfloat16* x, co
                           int32_t* dev_status, cudaStream_t stream) {
   const int K = p.kv_lora_rank + p.qk_rope_dim;
   const int ts = append_token_splits(p);
-  return launch_pdl(append_kernel, dim3(K / 8 * ts), dim3(256), kAppendSmem, stream, x, w, positions, page_table, cache,
-                    dev_status, p.batch, p.q_len, p.hidden_dim, p.kv_lora_rank, p.qk_rope_dim, p.num_pages,
-                    p.max_pages_per_seq, p.rope_theta, ts);
+  const int wide = append_wide(p) ? 1 : 0;
+  return launch_pdl(append_kernel, dim3(K / (wide ? 32 : 8) * ts), dim3(256), kAppendSmem, stream, x, w, positions, page_table,
+                    cache, dev_status, p.batch, p.q_len, p.hidden_dim, p.kv_lora_rank, p.qk_rope_dim, p.num_pages,
+                    p.max_pages_per_seq, p.rope_theta, ts, wide);
 }
 
 cudaError_t launch_absorb_plan(const transmla_params_t& p, int G, const __nv_bfloat16* q_nope,
@@ -323,10 +339,11 @@ cudaError_t launch_prologue(const transmla_params_t& p, int G, const __nv_bfloat
     attr_set = true;
   }
   const int ts = append_token_splits(p);
-  const int blocks = 1 + (p.kv_lora_rank + p.qk_rope_dim) / 8 * ts + p.num_heads * ((p.kv_lora_rank + 127) / 128);
+  const int wide = append_wide(p) ? 1 : 0;
+  const int blocks = 1 + (p.kv_lora_rank + p.qk_rope_dim) / (wide ? 32 : 8) * ts + p.num_heads * ((p.kv_lora_rank + 127) / 128);
   return launch_pdl(prologue_kernel, dim3(blocks), dim3(256), smem, stream, x, w_dkv_kr, page_table, cache, q_nope, q_pe,
                     w_uk, q_hat, seqlens, cum, plan, dev_status, p.batch, p.q_len, p.num_heads, p.hidden_dim,
-                    p.qk_nope_dim, p.qk_rope_dim, p.kv_lora_rank, p.num_pages, p.max_pages_per_seq, p.rope_theta, G, ts);
+                    p.qk_nope_dim, p.qk_rope_dim, p.kv_lora_rank, p.num_pages, p.max_pages_per_seq, p.rope_theta, G, ts, wide);
 }
 
 // ------------------------------------------------------------------------------------------------
