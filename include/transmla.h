@@ -219,8 +219,9 @@ transmla_status_t transmla_layer_decode_step(const transmla_params_t* params /* 
 /* Bytes of device staging transmla_decode_step_host needs for `params`. */
 size_t transmla_step_staging_bytes(const transmla_params_t* params /* host */);
 
-/* One whole decode step driven from host buffers: validates the tables on the host, copies this
- * step's inputs to the device (x, q_nope, q_pe, page_table, seqlens), runs transmla_decode_step,
+/* One whole decode step driven from host buffers: starts the copy of this step's inputs to the device
+ * (x, q_nope, q_pe, page_table, seqlens), validates the tables on the host meanwhile (a bad table ends the
+ * call before anything that uses the copies is launched), runs transmla_decode_step,
  * copies `out` (and `lse` if not NULL) back and waits for `stream`.  Weights and the cache stay
  * resident on the device.  When the host arrays are pinned (page-locked) the transfers are done by one
  * kernel each way that reads or writes the pinned memory directly; otherwise by one cudaMemcpyAsync per

@@ -289,11 +289,6 @@ transmla_status_t transmla_decode_step_host(const transmla_params_t* p, const vo
   if (p->qk_rope_dim > 0 && !h_q_pe) return TRANSMLA_ERR_NULL;
   if (!aligned(staging, kAlign)) return TRANSMLA_ERR_ALIGN;
   if (staging_bytes < transmla_step_staging_bytes(p)) return TRANSMLA_ERR_WORKSPACE;
-  st = transmla_validate_tables(p, h_page_table, h_seqlens);
-  if (st != TRANSMLA_OK) return st;
-  for (int b = 0; b < p->batch; ++b)
-    if (h_seqlens[b] < p->q_len) return TRANSMLA_ERR_RANGE;  // the step appends S tokens per sequence
-
   const size_t B = p->batch, S = p->q_len, H = p->num_heads;
   const size_t nx = B * S * p->hidden_dim * 2, nqn = B * S * H * p->qk_nope_dim * 2, nqp = B * S * H * p->qk_rope_dim * 2;
   const size_t npt = B * p->max_pages_per_seq * 4, nout = B * S * H * p->v_dim * 2, nlse = B * S * H * 4;
@@ -331,6 +326,13 @@ transmla_status_t transmla_decode_step_host(const transmla_params_t* p, const vo
     ok &= cudaMemsetAsync(d_st, 0, 4, s) == cudaSuccess;
   }
   if (!ok) return TRANSMLA_ERR_CUDA;
+  // The tables are checked on the host while the device already copies them: a bad table ends the call here,
+  // before anything that uses the staged copies is launched.
+  st = transmla_validate_tables(p, h_page_table, h_seqlens);
+  if (st != TRANSMLA_OK) return st;
+  for (int b = 0; b < p->batch; ++b)
+    if (h_seqlens[b] < p->q_len) return TRANSMLA_ERR_RANGE;  // the step appends S tokens per sequence
+  const bool out_pinned = is_pinned_host(h_out) && (h_lse == nullptr || is_pinned_host(h_lse));
   auto* dst = reinterpret_cast<int32_t*>(d_st);
   st = transmla_decode_step(p, d_x, d_qn, d_qp, reinterpret_cast<int32_t*>(d_pt), reinterpret_cast<int32_t*>(d_sl),
                             w_dkv_kr, w_uk, w_uv, cache, workspace, workspace_bytes,
@@ -338,7 +340,7 @@ transmla_status_t transmla_decode_step_host(const transmla_params_t* p, const vo
   if (st != TRANSMLA_OK) return st;
   int32_t dev_word = 0;
   int32_t* pinned_word = pinned_status_word();
-  if (pinned_word != nullptr && is_pinned_host(h_out) && (h_lse == nullptr || is_pinned_host(h_lse))) {
+  if (pinned_word != nullptr && out_pinned) {
     CopyList l = {};
     l.job[l.n++] = {d_out, h_out, nout};
     if (h_lse) l.job[l.n++] = {d_lse, h_lse, nlse};
