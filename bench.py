@@ -30,7 +30,7 @@ KERNELS_PER_STEP = 3      # prologue (append + absorb + plan), split-KV decode, 
 def workloads():
     from paper_2502_07864_b200 import synth
     w = {}
-    for B in (1, 4, 16, 64, 128):
+    for B in (1, 4, 16, 32, 64, 128):
         w[f'llama2-7b-mla_b{B}_8k'] = (synth.LLAMA2_7B, [8192] * B, 3)
     w['llama2-7b-mla_b16_8k'] = (synth.LLAMA2_7B, [8192] * 16, 2)
     w['llama2-7b-mla_ragged_b32'] = (synth.LLAMA2_7B, synth.uniform_seqlens(32, 1024, 32768, 4), 4)
