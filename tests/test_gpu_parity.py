@@ -294,7 +294,9 @@ def test_decode_step_from_host_buffers(pinned):
                                                # 48 and more new tokens: the large maps run on the tcgen05 kernel
                                                (synth.LLAMA2_7B, [70 + 3 * i for i in range(50)], 0),
                                                (synth.LLAMA2_7B, [64 + i for i in range(130)], 512),
-                                               (synth.QWEN25_72B, [66 + 5 * i for i in range(25)], 0)])
+                                               (synth.QWEN25_72B, [66 + 5 * i for i in range(25)], 0),
+                                               # more than 256 tokens: two token blocks per tile, the second nearly empty
+                                               (synth.LLAMA2_7B, [64 + (i % 7) for i in range(259)], 0)])
 def test_layer_decode_step(shape, seqlens, rq):
     B, S = len(seqlens), shape.S
     scale = gu.mla_scale(shape)
