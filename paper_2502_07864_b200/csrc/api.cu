@@ -67,6 +67,15 @@ __global__ void __launch_bounds__(256) copy_list_kernel(CopyList list) {
   }
 }
 
+// Blocks per array for the copy kernel: one per 16 KB of the largest array, between 24 and 128 (a few blocks
+// cannot keep enough reads in flight over PCIe once an array reaches a megabyte).
+int copy_blocks(const CopyList& l) {
+  unsigned long long most = 0;
+  for (int i = 0; i < l.n; ++i) most = l.job[i].bytes > most ? l.job[i].bytes : most;
+  const unsigned long long b = most / 16384;
+  return b < 24 ? 24 : b > 128 ? 128 : static_cast<int>(b);
+}
+
 bool is_pinned_host(const void* p) {
   cudaPointerAttributes a;
   if (cudaPointerGetAttributes(&a, p) != cudaSuccess) { cudaGetLastError(); return false; }
@@ -315,7 +324,7 @@ transmla_status_t transmla_decode_step_host(const transmla_params_t* p, const vo
     l.job[l.n++] = {h_page_table, d_pt, npt};
     l.job[l.n++] = {h_seqlens, d_sl, B * 4};
     l.zero_word = reinterpret_cast<int32_t*>(d_st);
-    copy_list_kernel<<<dim3(24, l.n), 256, 0, s>>>(l);
+    copy_list_kernel<<<dim3(copy_blocks(l), l.n), 256, 0, s>>>(l);
     ok &= cudaGetLastError() == cudaSuccess;
   } else {
     ok &= cudaMemcpyAsync(d_x, h_x, nx, cudaMemcpyHostToDevice, s) == cudaSuccess;
@@ -345,7 +354,7 @@ transmla_status_t transmla_decode_step_host(const transmla_params_t* p, const vo
     l.job[l.n++] = {d_out, h_out, nout};
     if (h_lse) l.job[l.n++] = {d_lse, h_lse, nlse};
     l.job[l.n++] = {d_st, pinned_word, 4};
-    copy_list_kernel<<<dim3(24, l.n), 256, 0, s>>>(l);
+    copy_list_kernel<<<dim3(copy_blocks(l), l.n), 256, 0, s>>>(l);
     ok &= cudaGetLastError() == cudaSuccess;
     ok &= cudaStreamSynchronize(s) == cudaSuccess;
     dev_word = *pinned_word;
