@@ -369,3 +369,22 @@ def test_many_serialized_launches_never_time_out(G):
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     assert (out.float() - first.float()).abs().max().item() <= 2e-2
+
+
+def test_dynamic_claims_when_some_partitions_find_nothing_left():
+    # A wide page table (capacity for 8K tokens) with short sequences: the library still picks 32+ partitions, most
+    # of the ones that own a page claim three at once, so the later ones find the sequence's counter past its end
+    # and must leave an empty partial (lse = -inf) that the combine skips.
+    shape = synth.LLAMA2_7B
+    seqlens = [640, 300, 64 * 7 + 1]
+    scale = gu.mla_scale(shape)
+    case = synth.make_decode_case(shape, seqlens, seed=29, nan_tails=True)
+    pad = torch.full((len(seqlens), 128 - case['page_table'].shape[1]), -1, dtype=torch.int32)
+    case['page_table'] = torch.cat([case['page_table'], pad], dim=1)
+    dev = gu.to_dev(case)
+    want, want_lse = gu.oracle_decode(shape, case, scale)
+    for _ in range(3):
+        out, lse, status, _, lay = gu.gpu_decode(shape, dev, scale, G=0)
+        assert status == 0 and lay.num_partitions >= 8 * len(seqlens)
+        gu.assert_close(lifts.f64(out), want, 'sparse dynamic claims')
+        gu.assert_lse_close(lifts.f64(lse), want_lse, 'sparse dynamic claims lse')
