@@ -184,6 +184,14 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
         for (int i = (lo & ~31) + lane * 32; i < hi; i += 32 * 32)
           asm volatile("prefetch.global.L1 [%0];" ::"l"(row + max(i, lo)));
       };
+      // The last sequence in which this partition owns pages: there it claims until the counter runs dry.  In the
+      // sequences before it (a partition that straddles two or more) it takes no more pages than the plan gave it,
+      // so that every sequence gets the share of CTA time that the plan meant it to have.
+      int last_home = pl.w;
+      if (dynamic) {
+        const int cw = cum[pl.w], cw1 = cum[pl.w + 1];
+        if (min(pl.y, cw1) <= max(pl.x, cw + kSegCost)) --last_home;
+      }
       for (int b = pl.z; b <= pl.w; ++b) {
         const int cb = cum[b], cb1 = cum[b + 1], L = seqlens[b];  // one round trip for the three of them
         const int c0s = cb + kSegCost;  // slot of page 0 of sequence b
@@ -202,8 +210,11 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
         // last one: it is exactly when the claim behind it is past the end (claims only grow).
         const int n_b = cb1 - c0s;
         int32_t* counter = next + static_cast<size_t>(rb) * B + b;
+        int left = b < last_home ? pg_hi - pg_lo : 0x7fffffff;  // claims this partition may still make here
+        const int take = min(kStages, left);
+        left -= take;
         int head = 0x7fffffff;
-        if (lane < kStages) head = atomicAdd(counter, 1);
+        if (lane < take) head = atomicAdd(counter, 1);
         prefetch_table(b, 0, n_b);  // in flight together with the claim
         int c0 = __shfl_sync(0xffffffffu, head, 0), c1 = __shfl_sync(0xffffffffu, head, 1), c2 = __shfl_sync(0xffffffffu, head, 2);
         { int t; if (c0 > c1) { t = c0; c0 = c1; c1 = t; } if (c1 > c2) { t = c1; c1 = c2; c2 = t; } if (c0 > c1) { t = c0; c0 = c1; c1 = t; } }
@@ -215,8 +226,8 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
         bool first = true;
         while (c0 < n_b) {
           int pend = 0x7fffffff;
-          const bool ahead = c2 < n_b;
-          if (ahead && lane == 0) pend = atomicAdd(counter, 1);
+          const bool ahead = c2 < n_b && left > 0;
+          if (ahead) { --left; if (lane == 0) pend = atomicAdd(counter, 1); }
           issue_page(b, c0, first, c1 >= n_b);
           first = false;
           c0 = c1;
