@@ -9,7 +9,8 @@ import numpy as np
 import pytest
 import torch
 
-from paper_2502_07864_b200 import synth
+from oracle import mla_oracle as orc
+from paper_2502_07864_b200 import binding, synth
 from tests import gpu_util as gu
 from tests import lifts
 
@@ -39,9 +40,9 @@ def sub_case(case, seqs, P=64):
     return out
 
 
-def check_sampled(shape, seqlens, seed, n_seq=3, n_heads=3):
+def check_sampled(shape, seqlens, seed, n_seq=3, n_heads=3, extra_pages=0):
     scale = gu.mla_scale(shape)
-    case = synth.make_decode_case(shape, seqlens, seed, device='cuda')
+    case = synth.make_decode_case(shape, seqlens, seed, device='cuda', extra_pages=extra_pages)
     out, lse, status, _, _ = gu.gpu_decode(shape, case, scale, G=0)
     assert status == 0
     assert torch.all(torch.isfinite(out.float()))
@@ -59,6 +60,7 @@ def check_sampled(shape, seqlens, seed, n_seq=3, n_heads=3):
     idx = tuple(np.array(only).T)
     gu.assert_close(got[idx], want[idx], f'sampled outputs B={B}')
     gu.assert_lse_close(got_lse[idx], want_lse[idx], 'sampled lse')
+    return case
 
 
 @pytest.mark.parametrize('B', [1, 4, 16, 64, 128])
@@ -78,6 +80,43 @@ def test_batch4_at_131072():
 def test_qwen_like_two_query_positions_batch64():
     seqlens = synth.uniform_seqlens(64, 2048, 8192, seed=5)
     check_sampled(synth.QWEN25_72B, seqlens, seed=5)
+
+
+def test_pool_larger_than_4_gib():
+    """Byte offsets into the pool need more than 32 bits: 62 000 pages of 73 728 bytes are 4.57 GB, and the seeded
+    permutation scatters the sequences' pages over all of it.  Decode is checked on sampled outputs, the append
+    on every row it writes and on every byte it must leave alone."""
+    shape, P = synth.LLAMA2_7B, synth.LLAMA2_7B.page_size
+    seqlens = [8192, 8192, 3000, 70, 8192, 8192]
+    case = check_sampled(shape, seqlens, seed=41, n_seq=2, n_heads=2, extra_pages=61000)
+    num_pages = case['cache'].shape[0]
+    assert num_pages * P * shape.row * 2 > 1 << 32
+    table = case['page_table'].cpu()
+    used = torch.cat([table[b, :(L + P - 1) // P] for b, L in enumerate(seqlens)])
+    assert int(used.max()) * P * shape.row * 2 > 1 << 32, 'the draw must place some page beyond 4 GiB'
+    # append the token at position L-1 of every sequence over what is there
+    positions = [L - 1 for L in seqlens]
+    ac = synth.make_append_case(shape, positions, 42, device='cuda')
+    before = case['cache'].clone()
+    params = binding.make_params(shape, len(seqlens), num_pages, table.shape[1], 1.0, num_partitions=1)
+    status = torch.zeros(1, dtype=torch.int32, device='cuda')
+    binding.transmla_latent_append(params, ac['x'], ac['w_dkv_kr'], ac['positions'], case['page_table'], case['cache'], status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    slots = [orc.append_slot(table[b].numpy(), positions[b], P) for b in range(len(seqlens))]
+    pg = torch.tensor([s[0] for s in slots]); off = torch.tensor([s[1] for s in slots])
+    got = lifts.f64(case['cache'][pg.cuda(), off.cuda()].cpu())                      # [B, r + dR]
+    small = np.zeros((len(seqlens), P, shape.row))                                 # one private page per sequence
+    small_table = np.full((len(seqlens), table.shape[1]), -1, dtype=np.int32)
+    for b_, pos in enumerate(positions):
+        small_table[b_, pos // P] = b_
+    orc.latent_append(lifts.f64(ac['x'][:, 0].cpu()), lifts.f64(ac['w_dkv_kr'].cpu()), positions, small_table, small,
+                      shape.r, page_size=P)
+    want = small[np.arange(len(seqlens)), off.numpy()]
+    assert np.all(np.abs(got - want) <= 2.0 ** -7 * np.abs(want) + 1e-3)
+    case['cache'][pg.cuda(), off.cuda()] = 0
+    before[pg.cuda(), off.cuda()] = 0
+    assert torch.equal(case['cache'].view(torch.int16), before.view(torch.int16))   # nothing else changed
 
 
 # ------------------------------------------------------------------ every output at full size, by closed forms
