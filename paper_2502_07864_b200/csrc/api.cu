@@ -165,6 +165,23 @@ static transmla_status_t check_decode_args(const transmla_params_t* p, const voi
   return check_device(nullptr);
 }
 
+// Host-side checks of a whole decode step, for callers inside the library that launch other kernels first.
+extern "C++" {
+namespace transmla {
+transmla_status_t validate_step_args(const transmla_params_t* p, const void* x, const void* q_nope, const void* q_pe,
+                                     const void* w_dkv_kr, const void* w_uk, const void* w_uv, const void* cache,
+                                     const int32_t* page_table, const int32_t* seqlens, void* workspace,
+                                     size_t workspace_bytes, const void* out, int32_t* dev_status) {
+  transmla_status_t st = check_shape(p, true);
+  if (st != TRANSMLA_OK) return st;
+  if (!x || !w_dkv_kr || !w_uv || !out) return TRANSMLA_ERR_NULL;
+  if (!aligned(x, 16) || !aligned(w_dkv_kr, 16) || !aligned(w_uv, 16) || !aligned(out, 16)) return TRANSMLA_ERR_ALIGN;
+  transmla_workspace_layout_t lay;
+  return check_decode_args(p, q_nope, q_pe, w_uk, cache, page_table, seqlens, workspace, workspace_bytes, dev_status, &lay);
+}
+}  // namespace transmla
+}  // extern "C++"
+
 // The split-KV kernel, bracketed by the caller's timing events when the profiling hook is armed.
 static transmla_status_t launch_split_kv(const transmla_params_t* p, const transmla_workspace_layout_t& lay,
                                          const void* cache, const int32_t* page_table, const int32_t* seqlens,

@@ -122,6 +122,10 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 // kernel before it in the stream is still draining: it calls pdl_trigger() at once (the kernel after it may
 // be scheduled as soon as SM resources allow) and pdl_wait() before the first access to anything an earlier
 // kernel of the stream may have produced or may still be reading.  Only weights are touched before the wait.
+// Pointers to anything but weights are therefore never declared `const __restrict__`: that pair tells the compiler
+// that the data cannot change while the kernel runs, which lets it issue the load above the wait (it did: the
+// combine read the plan's page total before the plan block had written it, once the kernels before it ran long
+// enough for its blocks to be resident that early).
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
@@ -156,6 +160,12 @@ __device__ __forceinline__ unsigned long long trace_now() {
 #define TRK_BEGIN(k) do { } while (0)
 #define TRK_END(k) do { } while (0)
 #endif
+
+// Every host-side check of transmla_decode_step, without launching anything.
+transmla_status_t validate_step_args(const transmla_params_t* p, const void* x, const void* q_nope, const void* q_pe,
+                                     const void* w_dkv_kr, const void* w_uk, const void* w_uv, const void* cache,
+                                     const int32_t* page_table, const int32_t* seqlens, void* workspace,
+                                     size_t workspace_bytes, const void* out, int32_t* dev_status);
 
 // Launchers (host).  Each enqueues on `stream` and returns the launch error, if any.
 bool dynamic_claims(const transmla_params_t& p, int G);  // whether the split-KV kernel hands pages out at run time

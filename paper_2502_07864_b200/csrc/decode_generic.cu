@@ -25,10 +25,10 @@ struct GenericCfg {
 
 template <int R, int DR>
 __global__ void __launch_bounds__(256, 1)
-decode_generic_kernel(const __nv_bfloat16* __restrict__ q_hat, const __nv_bfloat16* __restrict__ cache,
-                      const int32_t* __restrict__ page_table, const int32_t* __restrict__ seqlens,
-                      const int32_t* __restrict__ cum, const int32_t* __restrict__ plan,
-                      float* __restrict__ partial_o, float* __restrict__ partial_lse, int32_t* dev_status, int S, int H,
+decode_generic_kernel(const __nv_bfloat16* q_hat, const __nv_bfloat16* cache,
+                      const int32_t* page_table, const int32_t* seqlens,
+                      const int32_t* cum, const int32_t* plan,
+                      float* partial_o, float* partial_lse, int32_t* dev_status, int S, int H,
                       int num_pages, int max_pages, float scale_log2) {
   using C = GenericCfg<R, DR>;
   constexpr int K = C::K, KP = C::KP, KSW = C::KSW, NT = C::NT, SP = C::SP, PP = C::PP;

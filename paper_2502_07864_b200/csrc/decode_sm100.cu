@@ -75,10 +75,10 @@ enum { BAR_KV_FULL = 0, BAR_KV_EMPTY = kStages, BAR_Q_READY = 2 * kStages, BAR_S
 // ---------------------------------------------------------------------------------------------- kernel
 __global__ void __launch_bounds__(kThreads, 1)
 decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_constant__ CUtensorMap q_map,
-                    const int32_t* __restrict__ page_table, const int32_t* __restrict__ seqlens,
-                    const int32_t* __restrict__ cum, const int32_t* __restrict__ plan, float* __restrict__ partial_o,
-                    float* __restrict__ partial_lse, int32_t* dev_status, int S, int H, int num_pages, int max_pages,
-                    float scale_log2, int B, int dynamic, int32_t* __restrict__ next) {
+                    const int32_t* page_table, const int32_t* seqlens,
+                    const int32_t* cum, const int32_t* plan, float* partial_o,
+                    float* partial_lse, int32_t* dev_status, int S, int H, int num_pages, int max_pages,
+                    float scale_log2, int B, int dynamic, int32_t* next) {
   extern __shared__ unsigned char smem_unaligned[];
   const uint32_t raw = smem_u32(smem_unaligned);
   const uint32_t base = (raw + 1023u) & ~1023u;

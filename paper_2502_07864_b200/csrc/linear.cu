@@ -3,6 +3,7 @@
 // output features (see skinny_gemm.cuh).  One launch may hold two jobs (q^C and q^R share their input).
 #include <algorithm>
 
+#include "append_block.cuh"
 #include "common.cuh"
 #include "linear_args.cuh"
 #include "skinny_gemm.cuh"
@@ -11,12 +12,24 @@ namespace transmla {
 
 // MAXMT x 16 tokens per pass, NT x 8 output features per block.
 template <int MAXMT, int NT>
-__global__ void __launch_bounds__(256, 1) linear_kernel(LinearArgs a) {
+__global__ void __launch_bounds__(256, 1) linear_kernel(LinearArgs a, int32_t* dev_status) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   pdl_trigger();
   int nb = blockIdx.x, j = 0;
   const int blocks0 = a.job[0].N / (8 * NT) * a.t_splits;
-  if (a.n_jobs > 1 && nb >= blocks0) { nb -= blocks0; j = 1; }
+  const int blocks1 = a.n_jobs > 1 ? a.job[1].N / (8 * NT) * a.t_splits : 0;
+  if (nb >= blocks0 + blocks1) {  // the step's append: token (b, s) sits at pos_base[b] + pos_shift + s
+    const AppendJob& ap = a.append;
+    nb -= blocks0 + blocks1;
+    if (ap.wide)
+      append_block<1, 4>(ap.x, ap.w, a.pos_base, a.pos_shift, ap.page_table, ap.cache, dev_status, ap.B, a.S, ap.D, ap.r, ap.dR,
+                         ap.num_pages, ap.max_pages, a.theta, nb, ap.t_splits, smem_raw);
+    else
+      append_block<kAppendMaxMT, 1>(ap.x, ap.w, a.pos_base, a.pos_shift, ap.page_table, ap.cache, dev_status, ap.B, a.S, ap.D,
+                                    ap.r, ap.dR, ap.num_pages, ap.max_pages, a.theta, nb, ap.t_splits, smem_raw);
+    return;
+  }
+  if (nb >= blocks0) { nb -= blocks0; j = 1; }
   const LinearJob job = a.job[j];
   const int f_tiles = job.N / (8 * NT), f0 = (nb % f_tiles) * 8 * NT;
   const int t_chunk = (((a.M + a.t_splits - 1) / a.t_splits) + 15) & ~15;
@@ -31,14 +44,16 @@ __global__ void __launch_bounds__(256, 1) linear_kernel(LinearArgs a) {
   });
 }
 
-cudaError_t launch_linear(const LinearArgs& args, cudaStream_t stream) {
+cudaError_t launch_linear(const LinearArgs& args, int32_t* dev_status, cudaStream_t stream) {
   // 32 features per block when every job allows it (the activations are then read a quarter as often)
   bool wide = true;
   for (int j = 0; j < args.n_jobs; ++j) wide = wide && args.job[j].N % 32 == 0;
   const int per_block = wide ? 32 : 8;
   int blocks = 0;
   for (int j = 0; j < args.n_jobs; ++j) blocks += args.job[j].N / per_block * args.t_splits;
-  if (!wide) return launch_pdl(linear_kernel<8, 1>, dim3(blocks), dim3(256), skinny_gemm_smem(8, 1), stream, args);
+  blocks += args.append.blocks;  // short blocks at the end of the grid: they fill the last wave
+  static_assert(skinny_gemm_smem(8, 1) >= kAppendBlockSmem && skinny_gemm_smem(4, 4) >= kAppendBlockSmem, "append blocks fit");
+  if (!wide) return launch_pdl(linear_kernel<8, 1>, dim3(blocks), dim3(256), skinny_gemm_smem(8, 1), stream, args, dev_status);
   constexpr size_t smem = skinny_gemm_smem(4, 4);  // 64 KB: above the default limit
   static bool attr_set = false;
   if (!attr_set) {
@@ -46,7 +61,7 @@ cudaError_t launch_linear(const LinearArgs& args, cudaStream_t stream) {
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  return launch_pdl(linear_kernel<4, 4>, dim3(blocks), dim3(256), smem, stream, args);
+  return launch_pdl(linear_kernel<4, 4>, dim3(blocks), dim3(256), smem, stream, args, dev_status);
 }
 
 }  // namespace transmla
@@ -121,7 +136,7 @@ transmla_status_t transmla_layer_decode_step(const transmla_params_t* p, const t
   // One linear launch: the tcgen05 kernel where the shapes allow it, the mma.sync tiles otherwise.  The counters
   // of the tcgen05 kernel must be zero before its first launch of this call; every launch leaves them at zero.
   auto run_linear = [&](const LinearArgs& la) -> cudaError_t {
-    if (!linear_sm100_supported(la)) return launch_linear(la, s);
+    if (!linear_sm100_supported(la)) return launch_linear(la, dev_status, s);
     if (!counters_cleared) {
       cudaError_t e = cudaMemsetAsync(lin_counters, 0, counter_bytes, s);
       if (e != cudaSuccess) return e;
@@ -131,21 +146,48 @@ transmla_status_t transmla_layer_decode_step(const transmla_params_t* p, const t
   };
   const auto* xin = static_cast<const __nv_bfloat16*>(x);
 
+  transmla_status_t st = validate_step_args(p, x, q_nope, q_pe, w->w_dkv_kr, w->w_uk, w->w_uv, cache, page_table, seqlens,
+                                            workspace, workspace_bytes, attn, dev_status);
+  if (st != TRANSMLA_OK) return st;
+
   LinearArgs a = {};
   a.M = M; a.S = p->q_len; a.t_splits = token_splits(M); a.pos_base = seqlens; a.pos_shift = -p->q_len; a.theta = p->rope_theta;
+  // The append (Eq. 7 left) is one more linear map of x: where the layer's first launch runs on the mma.sync tiles
+  // its blocks ride in that launch, off the chain queries -> absorb -> attention; otherwise it stays in the
+  // attention step's prologue.
+  AppendJob ap = {};
+  ap.x = xin; ap.w = static_cast<const __nv_bfloat16*>(w->w_dkv_kr); ap.page_table = page_table;
+  ap.cache = static_cast<__nv_bfloat16*>(cache);
+  ap.B = p->batch; ap.D = D; ap.r = p->kv_lora_rank; ap.dR = p->qk_rope_dim; ap.num_pages = p->num_pages;
+  ap.max_pages = p->max_pages_per_seq; ap.t_splits = append_token_splits(*p); ap.wide = append_wide(*p) ? 1 : 0;
+  ap.blocks = (ap.r + ap.dR) / (ap.wide ? 32 : 8) * ap.t_splits;
+  bool appended = false;
+  auto with_append = [&](LinearArgs& la) {  // the first launch takes the append along if it can
+    if (!appended && !linear_sm100_supported(la)) { la.append = ap; appended = true; }
+  };
   if (low_rank) {  // c^Q = W_DQ x
     a.n_jobs = 1;
     a.job[0] = {xin, static_cast<const __nv_bfloat16*>(w->w_dq), cq, rq, D, 0};
+    with_append(a);
     if (run_linear(a) != cudaSuccess) return TRANSMLA_ERR_CUDA;
+    a.append = AppendJob{};
   }
   const __nv_bfloat16* qin = low_rank ? cq : xin;
   a.n_jobs = p->qk_rope_dim > 0 ? 2 : 1;  // q^C = W_UQ c^Q and q^R = RoPE(W_QR c^Q, t) in one launch
   a.job[0] = {qin, static_cast<const __nv_bfloat16*>(w->w_uq), q_nope, H * p->qk_nope_dim, Kq, 0};
   a.job[1] = {qin, static_cast<const __nv_bfloat16*>(w->w_qr), q_pe, H * p->qk_rope_dim, Kq, p->qk_rope_dim};
+  if (!low_rank) with_append(a);
   if (run_linear(a) != cudaSuccess) return TRANSMLA_ERR_CUDA;
+  a.append = AppendJob{};
 
-  transmla_status_t st = transmla_decode_step(p, x, q_nope, q_pe, page_table, seqlens, w->w_dkv_kr, w->w_uk, w->w_uv, cache,
-                                              workspace, workspace_bytes, attn, nullptr, dev_status, stream);
+  if (appended) {  // the new tokens' rows are in the cache (or on their way, earlier in the stream): attention only
+    st = transmla_mla_decode(p, q_nope, q_pe, w->w_uk, cache, page_table, seqlens, workspace, workspace_bytes, dev_status, stream);
+    if (st == TRANSMLA_OK)
+      st = transmla_mla_combine(p, workspace, workspace_bytes, w->w_uv, attn, nullptr, dev_status, stream);
+  } else {
+    st = transmla_decode_step(p, x, q_nope, q_pe, page_table, seqlens, w->w_dkv_kr, w->w_uk, w->w_uv, cache,
+                              workspace, workspace_bytes, attn, nullptr, dev_status, stream);
+  }
   if (st != TRANSMLA_OK) return st;
 
   a.n_jobs = 1;  // y = W_O [o_1; ...; o_h]

@@ -11,8 +11,18 @@ struct LinearJob {
   int N, K;
   int rope_d;               // > 0: consecutive blocks of rope_d output features are rotated (Eq. 1, d := rope_d)
 };
+// Append blocks riding in a launch of linear maps (Eq. 7 left is one more linear map of the same x): blocks
+// beyond those of the jobs run append_block.  blocks = 0: none.
+struct AppendJob {
+  const __nv_bfloat16* x;        // [B*S, D]
+  const __nv_bfloat16* w;        // [r + dR, D]
+  const int32_t* page_table;
+  __nv_bfloat16* cache;
+  int B, D, r, dR, num_pages, max_pages, t_splits, wide, blocks;
+};
 struct LinearArgs {
   LinearJob job[2];
+  AppendJob append;
   int n_jobs, M, S, t_splits;
   const int32_t* pos_base;  // position of token (b, s) = pos_base[b] + pos_shift + s (used by rotated jobs only)
   int pos_shift;

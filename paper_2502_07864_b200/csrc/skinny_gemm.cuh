@@ -28,7 +28,7 @@ constexpr size_t kAppendSmem = 8 * kAppendMaxMT * 16 * 8 * sizeof(float);  // 32
 
 // Partial products of one warp over its slice of the hidden dimension for tokens [t0, t0 + 16*MT).
 template <int MT, int UNROLL, int MAXMT, int NT>
-__device__ __forceinline__ void append_partial(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ wrow,
+__device__ __forceinline__ void append_partial(const __nv_bfloat16* x, const __nv_bfloat16* __restrict__ wrow,
                                                int D, int T, int t0, int k_lo, int slice, int g, int t4,
                                                float (&acc)[MAXMT][NT][4]) {
   const __nv_bfloat16* xr[MT][2];
@@ -70,7 +70,7 @@ constexpr size_t skinny_gemm_smem(int maxmt, int nt) { return static_cast<size_t
 // MAXMT: 16-token tiles per pass.  NT: 8-feature tiles per block; more of them re-read the activations less often,
 // which is what bounds these kernels once the weights are large (every block reads all its tokens' activations).
 template <int MAXMT = kAppendMaxMT, int NT = 1, class Epi>
-__device__ __forceinline__ void skinny_gemm_tile(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w,
+__device__ __forceinline__ void skinny_gemm_tile(const __nv_bfloat16* x, const __nv_bfloat16* __restrict__ w,
                                                  int K, int f0, int t_begin, int t_end, unsigned char* smem_raw, Epi epi) {
   float* red = reinterpret_cast<float*>(smem_raw);  // [8 warps][MAXMT*16 rows][8*NT]
   constexpr int kCols = 8 * NT;

@@ -11,6 +11,7 @@
 // sides load the 8 consecutive elements 8t .. 8t+7 of a 32-wide k window with one uint4 and feed words
 // (x, y) to one MMA and (z, w) to the next.  Where one operand comes from shared memory instead, it
 // is stored there in the matching order (kperm below).
+#include "append_block.cuh"
 #include "common.cuh"
 #include "skinny_gemm.cuh"
 
@@ -60,7 +61,7 @@ __device__ __forceinline__ int seq_of_page(const int32_t* cum, int B, int x) {
   return lo - 1;
 }
 
-__device__ void plan_block(const int32_t* __restrict__ seqlens, int B, int G, int RB, int32_t* cum, int32_t* plan,
+__device__ void plan_block(const int32_t* seqlens, int B, int G, int RB, int32_t* cum, int32_t* plan,
                            unsigned char* smem_raw) {
   __shared__ int warp_sums[8];
   __shared__ int carry;
@@ -123,8 +124,8 @@ __device__ void plan_block(const int32_t* __restrict__ seqlens, int B, int G, in
 constexpr int kAbsorbPitch = 128 + 8;
 constexpr int kAbsorbRows = 128;  // query rows staged per pass
 
-__device__ void absorb_block(const __nv_bfloat16* __restrict__ q_nope, const __nv_bfloat16* __restrict__ q_pe,
-                             const __nv_bfloat16* __restrict__ w_uk, __nv_bfloat16* __restrict__ q_hat, int BS, int H,
+__device__ void absorb_block(const __nv_bfloat16* q_nope, const __nv_bfloat16* q_pe,
+                             const __nv_bfloat16* __restrict__ w_uk, __nv_bfloat16* q_hat, int BS, int H,
                              int dn, int dR, int r, int h, int rt, unsigned char* smem_raw) {
   const int apitch = dn + 8;
   __nv_bfloat16* w_s = reinterpret_cast<__nv_bfloat16*>(smem_raw);  // [dn][kAbsorbPitch]
@@ -186,43 +187,11 @@ static size_t absorb_smem(int dn) {
   return (static_cast<size_t>(dn) * kAbsorbPitch + static_cast<size_t>(kAbsorbRows) * (dn + 8)) * sizeof(__nv_bfloat16);
 }
 
-// ------------------------------------------------------------------------------------------------
-// Latent append (Eq. 7 left): y = [W_DKV; W_KR] x, RoPE (Eq. 1) on y[r:], bf16, scatter to the page slot.
-// One block owns 8 consecutive output features (a RoPE pair never straddles blocks); its 8 warps
-// split the hidden dimension and meet in shared memory.  Tokens are the M dimension of the tiles.
-// Token (b, s) sits at position pos_base[b] + pos_shift + s.
-// ------------------------------------------------------------------------------------------------
-template <int MAXMT, int NT>
-__device__ void append_block(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w,
-                             const int32_t* __restrict__ pos_base, int pos_shift,
-                             const int32_t* __restrict__ page_table, __nv_bfloat16* __restrict__ cache,
-                             int32_t* dev_status, int B, int S, int D, int r, int dR, int num_pages, int max_pages,
-                             float theta, int nb, int t_splits, unsigned char* smem_raw) {
-  // block nb = (token split, feature tile): with many tokens the token range is cut so that more SMs take part
-  const int K = r + dR, f_tiles = K / (8 * NT), f0 = (nb % f_tiles) * 8 * NT;
-  const int t_chunk = (((B * S + t_splits - 1) / t_splits) + 15) & ~15;
-  const int t_begin = (nb / f_tiles) * t_chunk, t_end = min(B * S, t_begin + t_chunk);
-  skinny_gemm_tile<MAXMT, NT>(x, w, D, f0, t_begin, t_end, smem_raw, [&](int t, int pr, float re, float im) {
-    const int b = t / S, s = t % S;
-    const int pos = pos_base[b] + pos_shift + s;
-    const int pj = pos / kPage;
-    int page = -1;
-    if (pos >= 0 && pj < max_pages) page = page_table[static_cast<size_t>(b) * max_pages + pj];
-    if (page < 0 || page >= num_pages) {
-      set_status(dev_status, TRANSMLA_DEV_BAD_PAGE);
-      return;
-    }
-    const int f = f0 + pr * 2;
-    if (f >= r) rope_pair(re, im, pos, (f - r) >> 1, dR, theta);  // RoPE pair l of the decoupled key (Eq. 1)
-    *reinterpret_cast<uint32_t*>(cache + (static_cast<size_t>(page) * kPage + pos % kPage) * K + f) = pack_bf16(re, im);
-  });
-}
-
-__global__ void __launch_bounds__(256) append_kernel(const __nv_bfloat16* __restrict__ x,
+__global__ void __launch_bounds__(256) append_kernel(const __nv_bfloat16* x,
                                                      const __nv_bfloat16* __restrict__ w,
-                                                     const int32_t* __restrict__ positions,
-                                                     const int32_t* __restrict__ page_table,
-                                                     __nv_bfloat16* __restrict__ cache, int32_t* dev_status, int B,
+                                                     const int32_t* positions,
+                                                     const int32_t* page_table,
+                                                     __nv_bfloat16* cache, int32_t* dev_status, int B,
                                                      int S, int D, int r, int dR, int num_pages, int max_pages,
                                                      float theta, int t_splits, int wide) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -236,11 +205,11 @@ __global__ void __launch_bounds__(256) append_kernel(const __nv_bfloat16* __rest
 }
 
 // Absorb blocks followed by one plan block: everything transmla_mla_decode needs before the split-KV kernel.
-__global__ void __launch_bounds__(256) absorb_plan_kernel(const __nv_bfloat16* __restrict__ q_nope,
-                                                          const __nv_bfloat16* __restrict__ q_pe,
+__global__ void __launch_bounds__(256) absorb_plan_kernel(const __nv_bfloat16* q_nope,
+                                                          const __nv_bfloat16* q_pe,
                                                           const __nv_bfloat16* __restrict__ w_uk,
-                                                          __nv_bfloat16* __restrict__ q_hat,
-                                                          const int32_t* __restrict__ seqlens, int32_t* cum,
+                                                          __nv_bfloat16* q_hat,
+                                                          const int32_t* seqlens, int32_t* cum,
                                                           int32_t* plan, int B, int S, int H, int dn, int dR, int r,
                                                           int G) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -257,10 +226,10 @@ __global__ void __launch_bounds__(256) absorb_plan_kernel(const __nv_bfloat16* _
 // The whole prologue of a decode step in one launch: plan block, append blocks, absorb blocks.
 // The appended token of sequence b sits at seqlens[b] - S + s.
 __global__ void __launch_bounds__(256) prologue_kernel(
-    const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ w_dkv_kr,
-    const int32_t* __restrict__ page_table, __nv_bfloat16* __restrict__ cache, const __nv_bfloat16* __restrict__ q_nope,
-    const __nv_bfloat16* __restrict__ q_pe, const __nv_bfloat16* __restrict__ w_uk, __nv_bfloat16* __restrict__ q_hat,
-    const int32_t* __restrict__ seqlens, int32_t* cum, int32_t* plan, int32_t* dev_status, int B, int S, int H, int D,
+    const __nv_bfloat16* x, const __nv_bfloat16* __restrict__ w_dkv_kr,
+    const int32_t* page_table, __nv_bfloat16* cache, const __nv_bfloat16* q_nope,
+    const __nv_bfloat16* q_pe, const __nv_bfloat16* __restrict__ w_uk, __nv_bfloat16* q_hat,
+    const int32_t* seqlens, int32_t* cum, int32_t* plan, int32_t* dev_status, int B, int S, int H, int D,
     int dn, int dR, int r, int num_pages, int max_pages, float theta, int G, int t_splits, int wide) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   pdl_trigger();
@@ -289,10 +258,10 @@ constexpr int kPrologueMaxSmem = 144 * 1024;
 // Token splits of the append: one per 64 new tokens, at most 4.
 // With many new tokens a block takes 32 output features and 16 tokens (activations re-read a quarter as often
 // per feature, weights four times as often per token: 384 KB per block instead of 576 KB at 128 tokens).
-static bool append_wide(const transmla_params_t& p) {
+bool append_wide(const transmla_params_t& p) {
   return p.batch * p.q_len > 32 && (p.kv_lora_rank + p.qk_rope_dim) % 32 == 0 && p.kv_lora_rank % 2 == 0;
 }
-static int append_token_splits(const transmla_params_t& p) {
+int append_token_splits(const transmla_params_t& p) {
   const int T = p.batch * p.q_len;
   if (append_wide(p)) return (T + 15) / 16 > 32 ? 32 : (T + 15) / 16;
   return T <= 64 ? 1 : (T + 63) / 64 > 4 ? 4 : (T + 63) / 64;
@@ -361,11 +330,11 @@ constexpr int kCombineRows = 16;
 // kPrefetch: hold the first weight tile in registers from before the dependency wait (few blocks, latency
 // matters); otherwise load weights window by window and keep the register count low enough for two blocks per SM.
 template <bool kPrefetch>
-__global__ void __launch_bounds__(256, kPrefetch ? 1 : 2) combine_kernel(const int32_t* __restrict__ cum,
-                                                      const float* __restrict__ partial_o,
-                                                      const float* __restrict__ partial_lse,
+__global__ void __launch_bounds__(256, kPrefetch ? 1 : 2) combine_kernel(const int32_t* cum,
+                                                      const float* partial_o,
+                                                      const float* partial_lse,
                                                       const __nv_bfloat16* __restrict__ w_uv,
-                                                      __nv_bfloat16* __restrict__ out, float* __restrict__ lse_out,
+                                                      __nv_bfloat16* out, float* lse_out,
                                                       int B, int S, int H, int r, int dv, int G, int rows_per_block) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int pitch = r + 8;

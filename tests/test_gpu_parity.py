@@ -322,6 +322,42 @@ def test_layer_decode_step(shape, seqlens, rq):
     err, rel = gu.assert_close(lifts.f64(y), want, f'layer output rq={rq}')
 
 
+@pytest.mark.parametrize('shape,seqlens', [(synth.QWEN25_72B, [131, 700]), (synth.LLAMA2_7B, [300, 65, 1024])])
+def test_layer_step_repeated_on_a_poisoned_workspace(shape, seqlens):
+    """Nothing may be read before the kernel that produces it has finished.  From the second call on every kernel is
+    loaded and the launches overlap as far as they can, so a load issued ahead of its dependency wait meets whatever
+    the workspace held: it is filled with NaN bytes before every call, and every call must give the bits of the first
+    and meet the oracle."""
+    B, S = len(seqlens), shape.S
+    scale = gu.mla_scale(shape)
+    dc = synth.make_decode_case(shape, seqlens, 31)
+    ac = synth.make_append_case(shape, [L - S for L in seqlens], 32)
+    lw = synth.make_layer_weights(shape, 33)
+    weights = {k: v.cuda() for k, v in lw.items()}
+    weights.update(w_dkv_kr=ac['w_dkv_kr'].cuda(), w_uk=dc['w_uk'].cuda(), w_uv=dc['w_uv'].cuda())
+    params = binding.make_params(shape, B, dc['cache'].shape[0], dc['page_table'].shape[1], scale)
+    ws, _ = binding.alloc_workspace(params)
+    x, table, lens = ac['x'].cuda(), dc['page_table'].cuda(), dc['seqlens'].cuda()
+    outs = []
+    for it in range(6):
+        ws.fill_(0xff)
+        scratch = torch.full((binding.transmla_layer_scratch_bytes(params, 0),), 0xff, dtype=torch.uint8, device='cuda')
+        y = torch.full((B, S, shape.D), float('nan'), dtype=torch.bfloat16, device='cuda')
+        status = torch.zeros(1, dtype=torch.int32, device='cuda')
+        cache = dc['cache'].cuda()
+        torch.cuda.synchronize()
+        binding.transmla_layer_decode_step(params, weights, x, table, lens, cache, ws, scratch, y, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        outs.append(y.cpu())
+    for it in range(1, 6):
+        assert torch.equal(outs[it].view(torch.int16), outs[0].view(torch.int16)), f'call {it} differs from the first'
+    want = orc.mla_layer_decode(lifts.f64(ac['x']), lifts.f64(lw['w_uq']), lifts.f64(lw['w_qr']), lifts.f64(ac['w_dkv_kr']),
+                                lifts.f64(dc['w_uk']), lifts.f64(dc['w_uv']), lifts.f64(lw['w_o']), lifts.f64(dc['cache']),
+                                dc['page_table'].numpy(), seqlens, scale, shape.r)
+    gu.assert_close(lifts.f64(outs[0]), want, 'layer output on a poisoned workspace')
+
+
 # ------------------------------------------------------------------ pages claimed at run time (G = 0, many CTAs per sequence)
 @pytest.mark.parametrize('shape,seqlens', [(synth.LLAMA2_7B, [4096 + 17, 2100]), (synth.LLAMA2_7B, [8192]),
                                            (synth.LLAMA2_7B, [64 * 40, 64 * 41 + 1, 3000]),
