@@ -204,8 +204,10 @@ typedef struct {
 size_t transmla_layer_scratch_bytes(const transmla_params_t* params /* host */, int32_t q_lora_rank);
 
 /* The whole attention layer for the S newest tokens of every sequence, x [B, S, D] -> y [B, S, D] (device bf16):
- * queries (Eq. 8 right column, RoPE of q^R at position L_b - S + s), then transmla_decode_step (append, absorb,
- * split-KV decode, combine), then the output projection W_O (Eq. 9, last line).  The linear maps are skinny
+ * queries (Eq. 8 right column, RoPE of q^R at position L_b - S + s), then the steps of transmla_decode_step (append,
+ * absorb, split-KV decode, combine; with fewer than 48 new tokens the append's blocks run inside the layer's first
+ * launch of linear maps, beside the queries), then the output projection W_O (Eq. 9, last line).  Every host-side
+ * check of transmla_decode_step is made before anything is launched.  The linear maps are skinny
  * GEMMs with M = B*S that stream their weights once (mma.sync tiles; from 48 tokens on the large maps run as
  * TMA + tcgen05 tiles of 128 features with K cut into slices).  Needs D, H*dv (and r_q) multiples of 256; other rules
  * as for transmla_decode_step.  `scratch` is device memory of transmla_layer_scratch_bytes bytes, 256-byte
