@@ -319,7 +319,7 @@ def run_ours(args, name, shape, seqlens, seed):
     tflops = flops / (kernel_ms * 1e-3) / 1e12
     # ncu dram__bytes_read.sum + dram__bytes_write.sum of one split-KV launch on the default workload
     # (profiles/decode_sm100_llama2-7b_b16_8k.md); other workloads have no capture
-    traffic = 155.72e6 if name == 'llama2-7b-mla_b16_8k' and world == 1 else None
+    traffic = 155.63e6 if name == 'llama2-7b-mla_b16_8k' and world == 1 else None
     line = {
         'metric': METRIC, 'value': replicas.whole_job_rate(B * S, args.steps, ms_total), 'unit': 'tokens/s', 'n_gpus': world,
         'steps': args.steps, 'warmup': max(args.warmup, 3), 'ms_per_step': ms_step, 'higher_is_better': True,
