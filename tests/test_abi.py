@@ -77,3 +77,21 @@ def test_validate_tables_on_host():
     big = torch.tensor([[4, -1], [0, 2]], dtype=torch.int32)
     assert binding.transmla_validate_tables(p, big, torch.tensor([17, 128], dtype=torch.int32)) == 4
     assert binding.transmla_validate_tables(p, table, torch.tensor([-1, 0], dtype=torch.int32)) == 4
+
+
+def test_only_weights_are_declared_restrict_in_the_kernels():
+    """Every kernel starts before the kernel ahead of it in the stream has finished and waits later.  A pointer
+    declared const __restrict__ lets the compiler issue its loads above that wait, so only weights (which no
+    kernel of the stream writes) may carry the qualifier."""
+    import pathlib
+    import re
+    weights = {'w', 'w_uk', 'w_uv', 'w_dkv_kr', 'wrow'}
+    csrc = pathlib.Path(__file__).resolve().parent.parent / 'paper_2502_07864_b200' / 'csrc'
+    offenders = []
+    for f in sorted(csrc.iterdir()):
+        if f.suffix not in ('.cu', '.cuh'):
+            continue
+        for name in re.findall(r'__restrict__\s+(\w+)', f.read_text()):
+            if name not in weights:
+                offenders.append(f'{f.name}: {name}')
+    assert not offenders, offenders
