@@ -145,11 +145,29 @@ __device__ void absorb_block(const __nv_bfloat16* q_nope, const __nv_bfloat16* q
     const int rows = min(kAbsorbRows, BS - p0);
     const int rows16 = (rows + 15) & ~15;
     if (p0 > 0) __syncthreads();  // previous pass has consumed a_s
-    for (int i = tid; i < rows16 * chunks; i += 256) {
-      const int rr = i / chunks, c = i % chunks;
-      uint4 v = make_uint4(0, 0, 0, 0);
-      if (rr < rows) v = ld_u128(q_nope + (static_cast<size_t>(p0 + rr) * H + h) * dn + c * 8);
-      *reinterpret_cast<uint4*>(a_s + rr * apitch + c * 8) = v;
+    if (rows16 * chunks > 256) {
+      // many rows: eight 16-byte loads per thread in flight together (one at a time costs a trip to memory each)
+      for (int i0 = tid; i0 < rows16 * chunks; i0 += 256 * 8) {
+        uint4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int i = i0 + u * 256, rr = i / chunks, c = i % chunks;
+          v[u] = make_uint4(0, 0, 0, 0);
+          if (i < rows16 * chunks && rr < rows) v[u] = ld_u128(q_nope + (static_cast<size_t>(p0 + rr) * H + h) * dn + c * 8);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int i = i0 + u * 256, rr = i / chunks, c = i % chunks;
+          if (i < rows16 * chunks) *reinterpret_cast<uint4*>(a_s + rr * apitch + c * 8) = v[u];
+        }
+      }
+    } else {
+      for (int i = tid; i < rows16 * chunks; i += 256) {
+        const int rr = i / chunks, c = i % chunks;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (rr < rows) v = ld_u128(q_nope + (static_cast<size_t>(p0 + rr) * H + h) * dn + c * 8);
+        *reinterpret_cast<uint4*>(a_s + rr * apitch + c * 8) = v;
+      }
     }
     __syncthreads();
     for (int m0 = 0; m0 < rows16; m0 += 16) {
@@ -173,7 +191,23 @@ __device__ void absorb_block(const __nv_bfloat16* q_nope, const __nv_bfloat16* q
       }
     }
   }
-  if (rt == 0 && dR > 0) {
+  if (rt == 0 && dR > 0 && BS > 32 && dR % 8 == 0 && r % 8 == 0) {  // many rows: 16 bytes at a time, four copies in flight
+    const int vecs = dR / 8;
+    for (int i0 = tid; i0 < BS * vecs; i0 += 256 * 4) {
+      uint4 v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int i = i0 + u * 256, row = i / vecs, c = (i % vecs) * 8;
+        v[u] = make_uint4(0, 0, 0, 0);
+        if (i < BS * vecs) v[u] = ld_u128(q_pe + (static_cast<size_t>(row) * H + h) * dR + c);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int i = i0 + u * 256, row = i / vecs, c = (i % vecs) * 8;
+        if (i < BS * vecs) *reinterpret_cast<uint4*>(q_hat + (static_cast<size_t>(row) * H + h) * K + r + c) = v[u];
+      }
+    }
+  } else if (rt == 0 && dR > 0) {
     const int pairs = dR / 2;
     for (int i = tid; i < BS * pairs; i += 256) {
       const int row = i / pairs, c = (i % pairs) * 2;
