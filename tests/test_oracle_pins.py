@@ -412,6 +412,37 @@ def test_lifted_layer_reproduces_the_gqa_layer_output_token_by_token():
         assert np.abs(y[0, 0] - ref.reshape(-1) @ w_o.T).max() < 1e-10
 
 
+def test_layer_step_with_two_new_tokens_equals_two_single_token_steps():
+    # S = 2: token (b, s) sits at position L_b - S + s, the S latent rows are appended in that order and query
+    # s sees everything up to its own token.  One call with x[B, 2, D] must therefore give, token by token,
+    # what two successive single-token calls give on a cache that grows by one token per call.
+    rng = np.random.default_rng(23)
+    H, dn, dR, dv, r, D, P = 3, 4, 6, 5, 7, 12, 4
+    lens = [9, 4, 2]                                       # after the step; the last sequence starts empty
+    B = len(lens)
+    w = dict(w_uq=rng.standard_normal((H * dn, D)) / 3, w_qr=rng.standard_normal((H * dR, D)) / 3,
+             w_dkv_kr=rng.standard_normal((r + dR, D)) / 3, w_uk=rng.standard_normal((H, dn, r)) / 3,
+             w_uv=rng.standard_normal((H, dv, r)) / 3, w_o=rng.standard_normal((D, H * dv)) / 3)
+    table = np.array([[5, 1, 3], [0, 6, -1], [2, -1, -1]], dtype=np.int32)
+    base = np.full((7, P, r + dR), np.nan)
+    for b, L in enumerate(lens):                           # the L_b - 2 tokens cached before the step
+        for j in range(L - 2):
+            base[table[b, j // P], j % P] = rng.standard_normal(r + dR)
+    x = rng.standard_normal((B, 2, D))
+    args = lambda: (w['w_uq'], w['w_qr'], w['w_dkv_kr'], w['w_uk'], w['w_uv'], w['w_o'])
+    both = base.copy()
+    y2 = orc.mla_layer_decode(x, *args(), both, table, lens, 0.4, r, page_size=P)
+    one = base.copy()
+    y_first = orc.mla_layer_decode(x[:, :1], *args(), one, table, [L - 1 for L in lens], 0.4, r, page_size=P)
+    y_second = orc.mla_layer_decode(x[:, 1:], *args(), one, table, lens, 0.4, r, page_size=P)
+    assert np.abs(y2[:, 0] - y_first[:, 0]).max() < 1e-10
+    assert np.abs(y2[:, 1] - y_second[:, 0]).max() < 1e-10
+    assert np.array_equal(np.isnan(both), np.isnan(one)) and np.abs(np.nan_to_num(both - one)).max() < 1e-12
+    # the two tokens really differ in what they see: swapping the pair changes the result
+    swapped = orc.mla_layer_decode(x[:, ::-1], *args(), base.copy(), table, lens, 0.4, r, page_size=P)
+    assert np.abs(swapped[:, ::-1] - y2).max() > 1e-3
+
+
 def test_low_rank_queries_and_folded_output_projection():
     # Eq. 8 right: low-rank queries equal full-rank ones with W = W_U{Q,R} W_DQ; App. A.2.2: folding the block
     # diagonal of W_UV into W_O gives the same y from the latent-space outputs.
