@@ -23,9 +23,18 @@
  *     small, no sm_100 device) return an error code and launch nothing.  Problems only the device can
  *     see set bits in `*dev_status` (device int32, may be NULL; the caller zeroes it and reads it
  *     after synchronising) and never trap: a page-table entry outside [0, num_pages) is skipped
- *     (its tokens contribute nothing) and sets TRANSMLA_DEV_BAD_PAGE; a bounded wait that expired
- *     sets TRANSMLA_DEV_TIMEOUT and the affected results are unspecified.
- *   - Thread safety: no global mutable state except a cache of TMA descriptors guarded by a mutex.
+ *     (its tokens contribute nothing) and sets TRANSMLA_DEV_BAD_PAGE; a sequence length outside
+ *     [0, max_pages_per_seq * P] is clamped to that range (no look-up leaves the page table's row) and
+ *     sets TRANSMLA_DEV_BAD_LEN; a bounded wait that expired sets TRANSMLA_DEV_TIMEOUT and the affected
+ *     results are unspecified.
+ *   - Thread safety: entry points may be called from several host threads.  The library's own mutable
+ *     state is: per-device "already set" flags for kernel attributes and cluster-occupancy answers
+ *     (atomics; a race only repeats an idempotent runtime call), a per-device cache of the TMA
+ *     descriptors of the cache pool and of the workspace (guarded by a mutex), the per-thread timing
+ *     hook of transmla_profile_decode_kernel, a per-thread pinned status word used by
+ *     transmla_decode_step_host, and the built-in array of transmla_mla_attention_static, which all
+ *     calls on a device share (see the rule there).  Calls that use the same workspace, staging buffer or
+ *     output buffers must be ordered by the caller.
  */
 #ifndef TRANSMLA_H_
 #define TRANSMLA_H_
@@ -55,6 +64,7 @@ typedef enum {
  * internal waits were still pending (diagnostic only, no stable meaning) */
 #define TRANSMLA_DEV_BAD_PAGE 1
 #define TRANSMLA_DEV_TIMEOUT 2
+#define TRANSMLA_DEV_BAD_LEN 4
 
 typedef struct {
   int32_t hidden_dim;        /* D; used by the append only */
@@ -259,7 +269,8 @@ transmla_status_t transmla_decode_step_host(const transmla_params_t* params, con
  *     returns TRANSMLA_ERR_WORKSPACE and launches nothing.  The size grows with
  *     (num_partitions + B - 1) * S * H * r * 4 bytes; pass a smaller params->num_partitions to fit.
  *   - The first call on each device looks up the array's device address (with that device current)
- *     and remembers it; make that first call outside any stream capture.
+ *     and remembers it; make that first call outside any stream capture.  Device ordinals 0..63 are
+ *     served; on a device beyond that the call returns TRANSMLA_ERR_CUDA.
  *   - All calls on a device share the one array and it keeps whatever the previous call left there.
  *     A step never reads a region it has not itself written first, so no clearing is needed, but two
  *     calls whose kernels can overlap on the GPU (different streams, no ordering) race on it: issue
@@ -279,6 +290,16 @@ transmla_status_t transmla_mla_attention_static(const transmla_params_t* params 
  * (device int32, required), a second wait returns immediately and the kernel ends; the context stays
  * usable.  cycles_out (device int64[2], may be NULL) receives the SM cycles spent in the two waits. */
 transmla_status_t transmla_selftest_bounded_wait(int32_t* dev_status, long long* cycles_out, void* stream);
+
+/* Diagnostic: read-only streaming probe (no counterpart in the paper; it measures, it computes nothing).  Streams
+ * exactly the pages that the split-KV kernel of transmla_mla_decode reads for `params` - same grid, same split
+ * plan (taken from the workspace that a preceding transmla_mla_decode with the same `params` filled), same ring of
+ * TMA page loads - and discards them.  Timed with events around it, it gives the floor that launch, ramp-up and
+ * the memory system put under the split-KV kernel for this workload.  Only for r = 512, dR = 64
+ * (TRANSMLA_ERR_SHAPE otherwise).  Writes nothing but *dev_status (bad page indices are reported as usual). */
+transmla_status_t transmla_stream_probe(const transmla_params_t* params /* host */, const void* cache,
+                                        const int32_t* page_table, const void* workspace, size_t workspace_bytes,
+                                        int32_t* dev_status, void* stream);
 
 /* Timing hook: the next transmla_mla_decode issued by the calling thread records `start_event`
  * immediately before and `stop_event` immediately after its split-KV kernel on that call's stream

@@ -15,7 +15,7 @@ EXPORTS = ('transmla_workspace_layout', 'transmla_latent_append', 'transmla_mla_
            'transmla_validate_tables', 'transmla_step_staging_bytes', 'transmla_decode_step_host',
            'transmla_decode_step', 'transmla_profile_decode_kernel', 'transmla_status_string',
            'transmla_static_workspace_capacity', 'transmla_mla_attention_static', 'transmla_selftest_bounded_wait',
-           'transmla_layer_scratch_bytes', 'transmla_layer_decode_step')
+           'transmla_layer_scratch_bytes', 'transmla_layer_decode_step', 'transmla_stream_probe')
 
 
 class Params(ctypes.Structure):
@@ -72,6 +72,7 @@ def lib():
         L.transmla_static_workspace_capacity.restype = sz
         L.transmla_mla_attention_static.argtypes = [pp, vp, vp, vp, vp, vp, i32p, i32p, vp, vp, i32p, vp]
         L.transmla_selftest_bounded_wait.argtypes = [i32p, vp, vp]
+        L.transmla_stream_probe.argtypes = [pp, vp, i32p, vp, sz, i32p, vp]
         L.transmla_layer_scratch_bytes.argtypes = [pp, ctypes.c_int32]
         L.transmla_layer_scratch_bytes.restype = sz
         L.transmla_layer_decode_step.argtypes = [pp, ctypes.POINTER(LayerWeights), vp, i32p, i32p, vp, vp, sz, vp, sz, vp,
@@ -205,6 +206,13 @@ def transmla_layer_decode_step(params, weights, x, page_table, seqlens, cache, w
 def transmla_selftest_bounded_wait(dev_status, cycles_out=None, stream=None):
     _check(lib().transmla_selftest_bounded_wait(_ptr(dev_status), _ptr(cycles_out), _stream(stream)),
            'transmla_selftest_bounded_wait')
+
+
+def transmla_stream_probe(params, cache, page_table, workspace, dev_status=None, stream=None):
+    """Streams the pages of the split plan left in `workspace` by a preceding transmla_mla_decode and discards them."""
+    _check(lib().transmla_stream_probe(ctypes.byref(params), _ptr(cache), _ptr(page_table), _ptr(workspace),
+                                       workspace.numel() * workspace.element_size(), _ptr(dev_status), _stream(stream)),
+           'transmla_stream_probe')
 
 
 def transmla_profile_decode_kernel(start_event, stop_event):

@@ -214,7 +214,7 @@ transmla_status_t transmla_mla_decode(const transmla_params_t* p, const void* q_
                          static_cast<const __nv_bfloat16*>(q_pe), static_cast<const __nv_bfloat16*>(w_uk),
                          reinterpret_cast<__nv_bfloat16*>(ws + lay.q_hat_offset), seqlens,
                          reinterpret_cast<int32_t*>(ws + lay.cum_pages_offset),
-                         reinterpret_cast<int32_t*>(ws + lay.plan_offset), s) != cudaSuccess)
+                         reinterpret_cast<int32_t*>(ws + lay.plan_offset), dev_status, s) != cudaSuccess)
     return TRANSMLA_ERR_CUDA;
   return launch_split_kv(p, lay, cache, page_table, seqlens, ws, dev_status, s);
 }
@@ -237,6 +237,27 @@ transmla_status_t transmla_mla_combine(const transmla_params_t* p, const void* w
                                  reinterpret_cast<const float*>(ws + lay.partial_lse_offset),
                                  static_cast<const __nv_bfloat16*>(w_uv), static_cast<__nv_bfloat16*>(out), lse_out,
                                  dev_status, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? TRANSMLA_OK : TRANSMLA_ERR_CUDA;
+}
+
+transmla_status_t transmla_stream_probe(const transmla_params_t* p, const void* cache, const int32_t* page_table,
+                                        const void* workspace, size_t workspace_bytes, int32_t* dev_status,
+                                        void* stream) {
+  transmla_workspace_layout_t lay;
+  transmla_status_t st = transmla_workspace_layout(p, &lay);
+  if (st != TRANSMLA_OK) return st;
+  if (!decode_sm100_supported(*p)) return TRANSMLA_ERR_SHAPE;
+  if (!cache || !page_table || !workspace) return TRANSMLA_ERR_NULL;
+  if (!aligned(cache, 128) || !aligned(page_table, 4) || !aligned(workspace, kAlign) || !aligned(dev_status, 4))
+    return TRANSMLA_ERR_ALIGN;
+  if (workspace_bytes < lay.total_bytes) return TRANSMLA_ERR_WORKSPACE;
+  st = check_device(nullptr);
+  if (st != TRANSMLA_OK) return st;
+  const char* ws = static_cast<const char*>(workspace);
+  cudaError_t e = launch_stream_probe(*p, lay.num_partitions, static_cast<const __nv_bfloat16*>(cache), page_table,
+                                      reinterpret_cast<const int32_t*>(ws + lay.cum_pages_offset),
+                                      reinterpret_cast<const int32_t*>(ws + lay.plan_offset), dev_status,
+                                      static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? TRANSMLA_OK : TRANSMLA_ERR_CUDA;
 }
 

@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "transmla.h"
 
 namespace transmla {
@@ -20,6 +22,15 @@ constexpr float kLn2 = 0.6931471805599453f;
 
 __device__ __forceinline__ void set_status(int32_t* dev_status, int bit) {
   if (dev_status != nullptr) atomicOr(dev_status, bit);
+}
+
+// A sequence length outside [0, max_pages * P] cannot be honoured, the page table has no entries for it: it is
+// clamped, so that no look-up leaves the table's row, and reported through TRANSMLA_DEV_BAD_LEN.
+__device__ __forceinline__ int clamped_len(int L, int max_pages, int32_t* dev_status) {
+  const long long cap = static_cast<long long>(max_pages) * kPage;
+  if (L >= 0 && L <= cap) return L;
+  set_status(dev_status, TRANSMLA_DEV_BAD_LEN);
+  return L < 0 ? 0 : static_cast<int>(cap);
 }
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -130,6 +141,28 @@ __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.lau
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
+// Per-device host-side bookkeeping.  Function attributes (the dynamic shared memory limit) and occupancy answers
+// belong to one device, so what has been set or asked is remembered per device ordinal, in atomics: two host
+// threads that race through the first call both make the (idempotent) runtime call, nothing else.
+constexpr int kMaxDevices = 64;
+inline int current_device_slot() {  // the current device's ordinal, or -1 (then nothing is remembered)
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return -1; }
+  return dev >= 0 && dev < kMaxDevices ? dev : -1;
+}
+struct PerDeviceFlag {
+  std::atomic<int> value[kMaxDevices];
+};
+// Raises the kernel's dynamic shared memory limit on the current device, once per device.
+template <typename Kernel>
+cudaError_t ensure_dynamic_smem(Kernel kernel, int bytes, PerDeviceFlag& done) {
+  const int slot = current_device_slot();
+  if (slot >= 0 && done.value[slot].load(std::memory_order_acquire) != 0) return cudaSuccess;
+  const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess && slot >= 0) done.value[slot].store(1, std::memory_order_release);
+  return e;
+}
+
 template <typename... KArgs, typename... Args>
 cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args) {
   cudaLaunchConfig_t cfg = {};
@@ -145,22 +178,6 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
-// Optional kernel-level timeline (compile with -DTRANSMLA_TRACE): global-timer time of the first block start
-// and the last block end of each kernel, to see how the step's kernels overlap in a pipelined run.
-#ifdef TRANSMLA_TRACE
-extern __device__ unsigned long long g_ktrace[8][2];
-__device__ __forceinline__ unsigned long long trace_now() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-#define TRK_BEGIN(k) do { if (threadIdx.x == 0) atomicMin(&g_ktrace[k][0], trace_now()); } while (0)
-#define TRK_END(k) do { if (threadIdx.x == 0) atomicMax(&g_ktrace[k][1], trace_now()); } while (0)
-#else
-#define TRK_BEGIN(k) do { } while (0)
-#define TRK_END(k) do { } while (0)
-#endif
-
 // Every host-side check of transmla_decode_step, without launching anything.
 transmla_status_t validate_step_args(const transmla_params_t* p, const void* x, const void* q_nope, const void* q_pe,
                                      const void* w_dkv_kr, const void* w_uk, const void* w_uv, const void* cache,
@@ -171,7 +188,8 @@ transmla_status_t validate_step_args(const transmla_params_t* p, const void* x, 
 bool dynamic_claims(const transmla_params_t& p, int G);  // whether the split-KV kernel hands pages out at run time
 cudaError_t launch_absorb_plan(const transmla_params_t& p, int G, const __nv_bfloat16* q_nope,
                                const __nv_bfloat16* q_pe, const __nv_bfloat16* w_uk, __nv_bfloat16* q_hat,
-                               const int32_t* seqlens, int32_t* cum, int32_t* plan, cudaStream_t stream);
+                               const int32_t* seqlens, int32_t* cum, int32_t* plan, int32_t* dev_status,
+                               cudaStream_t stream);
 cudaError_t launch_prologue(const transmla_params_t& p, int G, const __nv_bfloat16* x, const __nv_bfloat16* w_dkv_kr,
                             const int32_t* page_table, __nv_bfloat16* cache, const __nv_bfloat16* q_nope,
                             const __nv_bfloat16* q_pe, const __nv_bfloat16* w_uk, __nv_bfloat16* q_hat,
@@ -189,6 +207,8 @@ cudaError_t launch_decode_sm100(const transmla_params_t& p, int G, const __nv_bf
                                 const __nv_bfloat16* cache, const int32_t* page_table, const int32_t* seqlens,
                                 const int32_t* cum, const int32_t* plan, float* partial_o, float* partial_lse,
                                 int32_t* dev_status, cudaStream_t stream);
+cudaError_t launch_stream_probe(const transmla_params_t& p, int G, const __nv_bfloat16* cache, const int32_t* page_table,
+                                const int32_t* cum, const int32_t* plan, int32_t* dev_status, cudaStream_t stream);
 cudaError_t launch_combine(const transmla_params_t& p, int G, const int32_t* cum, const float* partial_o,
                            const float* partial_lse, const __nv_bfloat16* w_uv, __nv_bfloat16* out, float* lse_out,
                            int32_t* dev_status, cudaStream_t stream);

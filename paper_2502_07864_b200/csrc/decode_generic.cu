@@ -57,7 +57,7 @@ decode_generic_kernel(const __nv_bfloat16* q_hat, const __nv_bfloat16* cache,
     const int c0 = cum[b] + kSegCost;  // slot of page 0 of sequence b
     const int pg_lo = max(pl.x, c0) - c0, pg_hi = min(pl.y, cum[b + 1]) - c0;
     if (pg_hi <= pg_lo) continue;
-    const int L = seqlens[b];
+    const int L = clamped_len(seqlens[b], max_pages, nullptr);  // the plan block has already reported a bad length
     const int slot = part + b;
     __syncthreads();  // previous segment fully done with shared memory
 
@@ -268,12 +268,8 @@ static cudaError_t launch_one(const transmla_params_t& p, int G, const __nv_bflo
                               int32_t* dev_status, cudaStream_t stream) {
   using C = GenericCfg<R, DR>;
   auto kern = decode_generic_kernel<R, DR>;
-  static bool attr_set = false;  // one flag per (R, DR) instantiation
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(C::smem_bytes));
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static PerDeviceFlag smem_set;  // zero-initialised; one slot per device
+  if (cudaError_t e = ensure_dynamic_smem(kern, static_cast<int>(C::smem_bytes), smem_set); e != cudaSuccess) return e;
   const int SH = p.q_len * p.num_heads;
   dim3 grid(G, (SH + kRowBlock - 1) / kRowBlock);
   return launch_pdl(kern, grid, dim3(256), C::smem_bytes, stream, q_hat, cache, page_table, seqlens, cum, plan, partial_o,

@@ -24,28 +24,6 @@
 namespace transmla {
 namespace sm100 {
 
-// Optional timeline instrumentation (compile with -DTRANSMLA_TRACE): clock64 stamps of one CTA's pipeline
-// events and the global-timer start/end of every CTA, read back with transmla_trace_dump().
-#ifdef TRANSMLA_TRACE
-__device__ long long g_trace[24][256];
-#define TR(ev, idx) do { if (blockIdx.x == 3 && blockIdx.y == 0 && (idx) < 256) g_trace[ev][idx] = clock64(); } while (0)
-#define TR_SMID() do { unsigned s_; asm volatile("mov.u32 %0, %%smid;" : "=r"(s_)); if (blockIdx.x < 256 && blockIdx.y == 0) g_trace[21][blockIdx.x] = s_; } while (0)
-#define TR_VAL(ev, v) do { if (blockIdx.x < 256 && blockIdx.y == 0) g_trace[ev][blockIdx.x] = (v); } while (0)
-#define TR_GLOBAL(ev) do { long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); if (blockIdx.x < 256 && blockIdx.y == 0) g_trace[ev][blockIdx.x] = t_; } while (0)
-#else
-#define TR(ev, idx) do { } while (0)
-#define TR_GLOBAL(ev) do { } while (0)
-#define TR_SMID() do { } while (0)
-#define TR_VAL(ev, v) do { } while (0)
-#endif
-
-#ifdef TRANSMLA_DBG
-__device__ int g_dbg[256][16];
-#define DBG(i, v) do { dbg_s[i] = (v); } while (0)
-#else
-#define DBG(i, v) do { } while (0)
-#endif
-
 constexpr int R = 512, DR = 64, K = R + DR;
 constexpr int kChunks = K / 64;                       // 9 sub-tiles of 64 columns (128 bytes) per page
 constexpr int kSubTileBytes = kPage * 128;            // 8192
@@ -94,13 +72,8 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int part = blockIdx.x, rb = blockIdx.y;
-#ifdef TRANSMLA_DBG
-  __shared__ volatile int dbg_s[16];
-  if (tid < 16) dbg_s[tid] = -1;
-#endif
   const int SH = S * H;
   pdl_trigger();
-  TRK_BEGIN(1);
 
   if (tid == 0) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&cache_map)) : "memory");
@@ -126,10 +99,8 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_base_s;
-  if (tid == 0) { TR(13, 0); TR_GLOBAL(15); TR_SMID(); }
   pdl_wait();  // the plan, the absorbed queries and the appended cache rows come from the kernel before this one
   const int4 pl = reinterpret_cast<const int4*>(plan)[part];
-  if (tid == 0) TR_GLOBAL(16);
   const bool has_home = pl.y > pl.x;
 
   if (has_home) {
@@ -142,12 +113,10 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
       auto acquire = [&](int gi) -> uint32_t {  // waits for the stage of ring item gi; returns its index
         const int stage = gi % kStages, use = gi / kStages;
         mbar_wait(bar(BAR_KV_EMPTY + stage), (use & 1) ^ 1, abort_flag, dev_status);
-        TR(0, gi);
         return stage;
       };
       auto issue_queries = [&](int b, int slot_code, int L) {
         const uint32_t stage = acquire(g);
-        if (g == 0 && lane == 0) TR_GLOBAL(17);
         if (!*abort_flag && elect_one()) {
           meta[g & (kMetaRing - 1)] = make_int4(ITEM_QUERIES, b, slot_code, L);
           mbar_arrive_expect_tx(bar(BAR_KV_FULL + stage), kChunks * kQTileBytes);
@@ -163,7 +132,6 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
         int idx = page_table[static_cast<size_t>(b) * max_pages + pj];
         const bool ok = idx >= 0 && idx < num_pages;
         if (!ok) { if (lane == 0) set_status(dev_status, TRANSMLA_DEV_BAD_PAGE); idx = 0; }
-        DBG(0, g); DBG(1, pj); DBG(2, (first ? 1 : 0) | (last ? 2 : 0));
         const uint32_t stage = acquire(g);
         if (!*abort_flag && elect_one()) {
           meta[g & (kMetaRing - 1)] = make_int4(ITEM_PAGE, pj, ok ? 1 : 0, (first ? 1 : 0) | (last ? 2 : 0));
@@ -193,7 +161,8 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
         if (min(pl.y, cw1) <= max(pl.x, cw + kSegCost)) --last_home;
       }
       for (int b = pl.z; b <= pl.w; ++b) {
-        const int cb = cum[b], cb1 = cum[b + 1], L = seqlens[b];  // one round trip for the three of them
+        const int cb = cum[b], cb1 = cum[b + 1];  // one round trip for the three of them
+        const int L = clamped_len(seqlens[b], max_pages, nullptr);  // the plan block has already reported a bad length
         const int c0s = cb + kSegCost;  // slot of page 0 of sequence b
         const int pg_lo = max(pl.x, c0s) - c0s, pg_hi = min(pl.y, cb1) - c0s;
         if (pg_hi <= pg_lo) continue;
@@ -235,7 +204,6 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
           c2 = ahead ? __shfl_sync(0xffffffffu, pend, 0) : 0x7fffffff;
         }
       }
-      if (lane == 0) TR_VAL(22, g);
       {  // closing item
         const uint32_t stage = acquire(g);
         if (elect_one()) {
@@ -258,7 +226,6 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
         // of the page before it is issued), and with a single barrier two of its phases could complete before this
         // wait looks at the first.  Per buffer the next phase needs the PV issued below to have completed.
         mbar_wait(bar(BAR_P_READY0 + (gp & 1)), (gp >> 1) & 1, abort_flag, dev_status);
-        TR(4, gr);
         tc_fence_after();
         const uint64_t a0 = smem_desc(base + kOffStage + stage * kStageBytes, kSubTileBytes, 1024);
         const uint64_t b0 = smem_desc(base + kOffP + (gp & 1) * kPBytes, 16, 1024);
@@ -277,7 +244,6 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
           tc_commit(bar(BAR_PV_DONE0 + (gp & 1)));
         }
         __syncwarp();
-        TR(5, gr);
       };
       while (true) {
         // a segment begins (or the ring ends): the softmax warps say which
@@ -290,11 +256,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
           const int stage = g % kStages, use = g / kStages;
           mbar_wait(bar(BAR_KV_FULL + stage), use & 1, abort_flag, dev_status);
           const int4 m = meta[g & (kMetaRing - 1)];
-          DBG(4, g); DBG(5, n); DBG(6, seg); DBG(7, m.w | (m.x << 8));
-          TR(1, g);
-          if (lane == 0) { if (n == 0) TR_GLOBAL(18); TR_GLOBAL(19); }
           if (n > 0) mbar_wait(bar(BAR_S_FREE), (n - 1) & 1, abort_flag, dev_status);
-          TR(2, g);
           tc_fence_after();
           const uint64_t k0 = smem_desc(base + kOffStage + stage * kStageBytes, 16, 1024);
 #pragma unroll
@@ -308,7 +270,6 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
           }
           if (elect_one()) tc_commit(bar(BAR_S_FULL));
           __syncwarp();
-          TR(3, g);
           if (pending) issue_pv(g - 1, n - 1, pending_first);
           pending = true;
           pending_first = (m.w & 1) != 0;
@@ -355,7 +316,7 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
         tc_fence_before();
         mbar_arrive(bar(BAR_Q_READY));
         asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (tid == 0) { mbar_arrive(bar(BAR_KV_EMPTY + stage)); TR(11, g); }
+        if (tid == 0) mbar_arrive(bar(BAR_KV_EMPTY + stage));
         ++g;
         return m;
       };
@@ -372,7 +333,6 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
           const int stage = g % kStages;
           mbar_wait(bar(BAR_KV_FULL + stage), (g / kStages) & 1, abort_flag, dev_status);
           const int4 pm = meta[g & (kMetaRing - 1)];
-          if (tid == 0) { DBG(8, g); DBG(9, n); DBG(10, pm.w | (pm.x << 8)); DBG(11, pm.y); }
           const int pj = pm.y;
           const bool page_ok = pm.z != 0;
           const int tok_end = page_ok ? n_vis - pj * kPage : 0;           // tokens [0, tok_end) of the page are visible
@@ -380,16 +340,13 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
           const bool first = (pm.w & 1) != 0;
           const int buf = n & 1;
 
-          if (tid == 0) TR(6, g);
           mbar_wait(bar(BAR_S_FULL), n & 1, abort_flag, dev_status);
-          if (tid == 0) TR(7, g);
           tc_fence_after();
           uint32_t sq[16];  // this warp's 16 tokens of its row
           tmem_ld16(tmem + lane_base + kColS + warp * 16, sq);
           tc_wait_ld();
           tc_fence_before();
           mbar_arrive(bar(BAR_S_FREE));
-          if (tid == 0) TR(8, g);
           {
             float pmax = -INFINITY;
 #pragma unroll
@@ -471,7 +428,6 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
           fence_proxy_async();
           tc_fence_before();
           mbar_arrive(bar(BAR_P_READY0 + buf));
-          if (tid == 0) TR(9, g);
           ++g; ++n;
         }
 
@@ -490,7 +446,6 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
         // The queries of the next segment go to tensor memory now (every QK^T of this segment has completed), so
         // that its first QK^T runs while this segment's result is written out.
         seg_meta = open_segment();
-        if (tid == 0) { TR(12, g); TR_GLOBAL(20); }
         const int n_last = n - 1;
         mbar_wait(bar(BAR_PV_DONE0 + (n_last & 1)), (n_last >> 1) & 1, abort_flag, dev_status);
         tc_fence_after();
@@ -512,17 +467,10 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
         }
         tc_fence_before();
         asm volatile("bar.sync 1, 128;" ::: "memory");  // inv_l and the row sums are reused by the next segment
-        if (tid == 0) TR(14, g);
       }
     }
   }
 
-  if (tid == 0) { TR(13, 1); TR_GLOBAL(10); }
-#ifdef TRANSMLA_DBG
-  __syncthreads();
-  if (*abort_flag && tid < 16 && blockIdx.x < 256 && blockIdx.y == 0) g_dbg[blockIdx.x][tid] = dbg_s[tid];
-#endif
-  TRK_END(1);
   // ---- teardown: everyone arrives, tensor memory is returned
   tc_fence_before();
   __syncthreads();
@@ -534,15 +482,6 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
 
 // ---------------------------------------------------------------------------------------------- host
 }  // namespace sm100
-
-#ifdef TRANSMLA_DBG
-extern "C" int transmla_dbg_dump(int* host) { return static_cast<int>(cudaMemcpyFromSymbol(host, sm100::g_dbg, sizeof(int) * 256 * 16)); }
-#endif
-#ifdef TRANSMLA_TRACE
-extern "C" int transmla_trace_dump(long long* host) {
-  return static_cast<int>(cudaMemcpyFromSymbol(host, sm100::g_trace, sizeof(long long) * 24 * 256));
-}
-#endif
 
 bool decode_sm100_supported(const transmla_params_t& p) { return p.kv_lora_rank == sm100::R && p.qk_rope_dim == sm100::DR; }
 
@@ -559,34 +498,16 @@ cudaError_t launch_decode_sm100(const transmla_params_t& p, int G, const __nv_bf
                                 const int32_t* cum, const int32_t* plan, float* partial_o, float* partial_lse,
                                 int32_t* dev_status, cudaStream_t stream) {
   using namespace sm100;
-  auto encode = encode_fn();
-  if (encode == nullptr) return cudaErrorNotSupported;
   // The pool as a 2-D tensor [num_pages * 64 rows, 576 columns]; one box = 64 rows x 64 columns (128 bytes),
-  // written to shared memory with the 128-byte swizzle the MMA descriptors expect.
-  CUtensorMap map;
-  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(K), static_cast<cuuint64_t>(p.num_pages) * kPage};
-  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(K) * sizeof(__nv_bfloat16)};
-  const cuuint32_t box[2] = {64, kPage};
-  const cuuint32_t elem_strides[2] = {1, 1};
-  if (encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(cache), dims, strides, box, elem_strides,
-             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-    return cudaErrorInvalidValue;
-  // The absorbed queries as a 2-D tensor [B*S*H rows, 576 columns]; one box = 32 rows x 64 columns.
-  CUtensorMap qmap;
+  // written to shared memory with the 128-byte swizzle the MMA descriptors expect.  The absorbed queries as a
+  // 2-D tensor [B*S*H rows, 576 columns]; one box = 32 rows x 64 columns.
+  CUtensorMap map, qmap;
   const int SH = p.q_len * p.num_heads;
-  const cuuint64_t qdims[2] = {static_cast<cuuint64_t>(K), static_cast<cuuint64_t>(p.batch) * SH};
-  const cuuint32_t qbox[2] = {64, kRowBlock};
-  if (encode(&qmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(q_hat), qdims, strides, qbox,
-             elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+  if (!tensor_map_2d(&map, cache, static_cast<uint64_t>(p.num_pages) * kPage, K, kPage) ||
+      !tensor_map_2d(&qmap, q_hat, static_cast<uint64_t>(p.batch) * SH, K, kRowBlock))
     return cudaErrorInvalidValue;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(decode_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static PerDeviceFlag smem_set;  // zero-initialised; one slot per device
+  if (cudaError_t e = ensure_dynamic_smem(decode_sm100_kernel, kSmemBytes, smem_set); e != cudaSuccess) return e;
   dim3 grid(G, (SH + kRowBlock - 1) / kRowBlock);
   int32_t* next = const_cast<int32_t*>(cum) + 3 * p.batch + 1;  // page counters, zeroed by the plan
   return launch_pdl(decode_sm100_kernel, grid, dim3(kThreads), static_cast<size_t>(kSmemBytes), stream, map, qmap,

@@ -55,12 +55,8 @@ cudaError_t launch_linear(const LinearArgs& args, int32_t* dev_status, cudaStrea
   static_assert(skinny_gemm_smem(8, 1) >= kAppendBlockSmem && skinny_gemm_smem(4, 4) >= kAppendBlockSmem, "append blocks fit");
   if (!wide) return launch_pdl(linear_kernel<8, 1>, dim3(blocks), dim3(256), skinny_gemm_smem(8, 1), stream, args, dev_status);
   constexpr size_t smem = skinny_gemm_smem(4, 4);  // 64 KB: above the default limit
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(linear_kernel<4, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static PerDeviceFlag smem_set;  // zero-initialised; one slot per device
+  if (cudaError_t e = ensure_dynamic_smem(linear_kernel<4, 4>, static_cast<int>(smem), smem_set); e != cudaSuccess) return e;
   return launch_pdl(linear_kernel<4, 4>, dim3(blocks), dim3(256), smem, stream, args, dev_status);
 }
 

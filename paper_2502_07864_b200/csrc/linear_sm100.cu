@@ -319,15 +319,7 @@ linear_sm100_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_con
 }
 
 static bool encode_2d(CUtensorMap* map, const void* ptr, int rows, int cols, int box_rows) {
-  auto encode = encode_fn();
-  if (encode == nullptr) return false;
-  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
-  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(cols) * sizeof(__nv_bfloat16)};
-  const cuuint32_t box[2] = {kLinBK, static_cast<cuuint32_t>(box_rows)};
-  const cuuint32_t elem_strides[2] = {1, 1};
-  return encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, elem_strides,
-                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return tensor_map_2d(map, ptr, static_cast<uint64_t>(rows), static_cast<uint32_t>(cols), static_cast<uint32_t>(box_rows), kLinBK);
 }
 
 }  // namespace sm100
@@ -394,12 +386,8 @@ cudaError_t launch_linear_sm100(const LinearArgs& a, float* partial, int32_t* co
   p.splits = linear_sm100_splits(tiles, p.K);
   p.pos_base = a.pos_base; p.pos_shift = a.pos_shift; p.theta = a.theta;
   p.partial = partial; p.counters = counters;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(linear_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kLinSmemBytes);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static PerDeviceFlag smem_set;  // zero-initialised; one slot per device
+  if (cudaError_t e = ensure_dynamic_smem(linear_sm100_kernel, kLinSmemBytes, smem_set); e != cudaSuccess) return e;
   const int token_blocks = (a.M + kLinMaxT - 1) / kLinMaxT;
   // The K slices of a tile are launched as one thread-block cluster (they are neighbours in blockIdx.x); they then
   // meet through distributed shared memory and need neither the scratch buffer nor the counters.  All clusters have
@@ -416,17 +404,20 @@ cudaError_t launch_linear_sm100(const LinearArgs& a, float* partial, int32_t* co
   attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
   cfg.attrs = attr;
   p.cluster = 0;
-  static int max_clusters[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};  // co-resident clusters of each size, asked once
+  static PerDeviceFlag max_clusters[9];  // co-resident clusters of each size on each device, asked once (0 = not yet)
+  const int slot = current_device_slot();
   for (int s = p.splits < 8 ? p.splits : 8; s >= 2 && !p.cluster; --s) {
     attr[1].val.clusterDim.x = s;
     cfg.gridDim = dim3(tiles * s, token_blocks);
     cfg.numAttrs = 2;
-    if (max_clusters[s] == 0) {
+    int fit = slot >= 0 ? max_clusters[s].value[slot].load(std::memory_order_acquire) : 0;
+    if (fit == 0) {
       int n = 0;
       if (cudaOccupancyMaxActiveClusters(&n, linear_sm100_kernel, &cfg) != cudaSuccess) { cudaGetLastError(); n = -1; }
-      max_clusters[s] = n > 0 ? n : -1;
+      fit = n > 0 ? n : -1;
+      if (slot >= 0) max_clusters[s].value[slot].store(fit, std::memory_order_release);
     }
-    if (max_clusters[s] >= tiles * token_blocks) { p.cluster = 1; p.splits = s; }
+    if (fit >= tiles * token_blocks) { p.cluster = 1; p.splits = s; }
   }
   if (!p.cluster) {
     cfg.gridDim = dim3(tiles * p.splits, token_blocks);

@@ -17,27 +17,6 @@
 
 namespace transmla {
 
-#ifdef TRANSMLA_TRACE
-__device__ unsigned long long g_ktrace[8][2];
-__device__ unsigned long long g_ctrace[16][1024];
-extern "C" int transmla_ctrace_dump(unsigned long long* host) { return static_cast<int>(cudaMemcpyFromSymbol(host, g_ctrace, sizeof(g_ctrace))); }
-#define TRC(ev) do { if (threadIdx.x == 0) { g_ctrace[ev][(blockIdx.y * gridDim.x + blockIdx.x) & 1023] = trace_now(); g_ctrace[4 + ev][(blockIdx.y * gridDim.x + blockIdx.x) & 1023] = clock64(); } } while (0)
-extern "C" int transmla_ktrace_dump(unsigned long long* host, int reset) {
-  int e = static_cast<int>(cudaMemcpyFromSymbol(host, g_ktrace, sizeof(g_ktrace)));
-  if (reset) {
-    unsigned long long init[8][2];
-    for (int i = 0; i < 8; ++i) { init[i][0] = ~0ull; init[i][1] = 0; }
-    cudaMemcpyToSymbol(g_ktrace, init, sizeof(init));
-  }
-  return e;
-}
-#define TRCK(ev) do { if (threadIdx.x == 0) g_ctrace[ev][(blockIdx.y * gridDim.x + blockIdx.x) & 1023] = clock64(); } while (0)
-#else
-#define TRC(ev) do { } while (0)
-#define TRCK(ev) do { } while (0)
-#endif
-
-
 // Position, inside its 32-wide window, at which element p must sit in shared memory so that ldmatrix
 // hands out the fragment that pairs with a uint4 global load of the other operand.
 __device__ __forceinline__ int kperm(int p) { return ((p & 7) >> 1) * 8 + (p >> 3) * 2 + (p & 1); }
@@ -61,8 +40,8 @@ __device__ __forceinline__ int seq_of_page(const int32_t* cum, int B, int x) {
   return lo - 1;
 }
 
-__device__ void plan_block(const int32_t* seqlens, int B, int G, int RB, int32_t* cum, int32_t* plan,
-                           unsigned char* smem_raw) {
+__device__ void plan_block(const int32_t* seqlens, int B, int G, int RB, int max_pages, int32_t* cum, int32_t* plan,
+                           int32_t* dev_status, unsigned char* smem_raw) {
   __shared__ int warp_sums[8];
   __shared__ int carry;
   int32_t* cum_s = reinterpret_cast<int32_t*>(smem_raw);  // [B+1] when B < kPlanSmemSeqs
@@ -74,7 +53,7 @@ __device__ void plan_block(const int32_t* seqlens, int B, int G, int RB, int32_t
   for (int base = 0; base < B; base += 256) {
     const int b = base + tid;
     int n = 0;
-    if (b < B) { int L = seqlens[b]; n = L > 0 ? (L + kPage - 1) / kPage + kSegCost : 0; }
+    if (b < B) { const int L = clamped_len(seqlens[b], max_pages, dev_status); n = L > 0 ? (L + kPage - 1) / kPage + kSegCost : 0; }
     int v = n;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) { int t = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += t; }
@@ -244,8 +223,8 @@ __global__ void __launch_bounds__(256) absorb_plan_kernel(const __nv_bfloat16* q
                                                           const __nv_bfloat16* __restrict__ w_uk,
                                                           __nv_bfloat16* q_hat,
                                                           const int32_t* seqlens, int32_t* cum,
-                                                          int32_t* plan, int B, int S, int H, int dn, int dR, int r,
-                                                          int G) {
+                                                          int32_t* plan, int32_t* dev_status, int B, int S, int H,
+                                                          int dn, int dR, int r, int G, int max_pages) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   pdl_trigger();
   const int r_tiles = (r + 127) / 128;
@@ -253,7 +232,7 @@ __global__ void __launch_bounds__(256) absorb_plan_kernel(const __nv_bfloat16* q
   if (static_cast<int>(blockIdx.x) < n_absorb) {
     absorb_block(q_nope, q_pe, w_uk, q_hat, B * S, H, dn, dR, r, blockIdx.x / r_tiles, blockIdx.x % r_tiles, smem_raw);
   } else {
-    plan_block(seqlens, B, G, (S * H + kRowBlock - 1) / kRowBlock, cum, plan, smem_raw);
+    plan_block(seqlens, B, G, (S * H + kRowBlock - 1) / kRowBlock, max_pages, cum, plan, dev_status, smem_raw);
   }
 }
 
@@ -267,12 +246,11 @@ __global__ void __launch_bounds__(256) prologue_kernel(
     int dn, int dR, int r, int num_pages, int max_pages, float theta, int G, int t_splits, int wide) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   pdl_trigger();
-  TRK_BEGIN(0);
   const int n_append = (r + dR) / (wide ? 32 : 8) * t_splits;
   const int r_tiles = (r + 127) / 128;
   const int bid = static_cast<int>(blockIdx.x) - 1;
   if (bid < 0) {
-    plan_block(seqlens, B, G, (S * H + kRowBlock - 1) / kRowBlock, cum, plan, smem_raw);
+    plan_block(seqlens, B, G, (S * H + kRowBlock - 1) / kRowBlock, max_pages, cum, plan, dev_status, smem_raw);
   } else if (bid < n_append) {
     if (wide)
       append_block<1, 4>(x, w_dkv_kr, seqlens, -S, page_table, cache, dev_status, B, S, D, r, dR, num_pages, max_pages,
@@ -284,7 +262,6 @@ __global__ void __launch_bounds__(256) prologue_kernel(
     const int a = bid - n_append;
     absorb_block(q_nope, q_pe, w_uk, q_hat, B * S, H, dn, dR, r, a / r_tiles, a % r_tiles, smem_raw);
   }
-  TRK_END(0);
 }
 
 constexpr int kPrologueMaxSmem = 144 * 1024;
@@ -314,18 +291,16 @@ cudaError_t launch_append(const transmla_params_t& p, const __nv_bfloat16* x, co
 
 cudaError_t launch_absorb_plan(const transmla_params_t& p, int G, const __nv_bfloat16* q_nope,
                                const __nv_bfloat16* q_pe, const __nv_bfloat16* w_uk, __nv_bfloat16* q_hat,
-                               const int32_t* seqlens, int32_t* cum, int32_t* plan, cudaStream_t stream) {
+                               const int32_t* seqlens, int32_t* cum, int32_t* plan, int32_t* dev_status,
+                               cudaStream_t stream) {
   size_t smem = absorb_smem(p.qk_nope_dim);
   if (smem < kPlanSmemSeqs * sizeof(int32_t)) smem = kPlanSmemSeqs * sizeof(int32_t);
-  static bool attr_set = false;  // above the default dynamic shared memory limit
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(absorb_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPrologueMaxSmem);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static PerDeviceFlag smem_set;  // zero-initialised; one slot per device
+  if (cudaError_t e = ensure_dynamic_smem(absorb_plan_kernel, kPrologueMaxSmem, smem_set); e != cudaSuccess) return e;
   const int blocks = p.num_heads * ((p.kv_lora_rank + 127) / 128) + 1;
   return launch_pdl(absorb_plan_kernel, dim3(blocks), dim3(256), smem, stream, q_nope, q_pe, w_uk, q_hat, seqlens, cum,
-                    plan, p.batch, p.q_len, p.num_heads, p.qk_nope_dim, p.qk_rope_dim, p.kv_lora_rank, G);
+                    plan, dev_status, p.batch, p.q_len, p.num_heads, p.qk_nope_dim, p.qk_rope_dim, p.kv_lora_rank, G,
+                    p.max_pages_per_seq);
 }
 
 cudaError_t launch_prologue(const transmla_params_t& p, int G, const __nv_bfloat16* x, const __nv_bfloat16* w_dkv_kr,
@@ -335,12 +310,8 @@ cudaError_t launch_prologue(const transmla_params_t& p, int G, const __nv_bfloat
                             cudaStream_t stream) {
   size_t smem = absorb_smem(p.qk_nope_dim);
   if (smem < kAppendSmem) smem = kAppendSmem;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(prologue_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPrologueMaxSmem);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static PerDeviceFlag smem_set;  // zero-initialised; one slot per device
+  if (cudaError_t e = ensure_dynamic_smem(prologue_kernel, kPrologueMaxSmem, smem_set); e != cudaSuccess) return e;
   const int ts = append_token_splits(p);
   const int wide = append_wide(p) ? 1 : 0;
   const int blocks = 1 + (p.kv_lora_rank + p.qk_rope_dim) / (wide ? 32 : 8) * ts + p.num_heads * ((p.kv_lora_rank + 127) / 128);
@@ -375,7 +346,6 @@ __global__ void __launch_bounds__(256, kPrefetch ? 1 : 2) combine_kernel(const i
   __nv_bfloat16* o_hi = reinterpret_cast<__nv_bfloat16*>(smem_raw);  // [16][pitch]
   __nv_bfloat16* o_lo = o_hi + kCombineRows * pitch;                 // [16][pitch]
   pdl_trigger();
-  TRK_BEGIN(2);
   const int h = blockIdx.x, bs0 = blockIdx.y * rows_per_block;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int SH = S * H, BS = B * S;
@@ -513,7 +483,6 @@ __global__ void __launch_bounds__(256, kPrefetch ? 1 : 2) combine_kernel(const i
     if (g + 8 < rows_per_block && bs_b < BS)
       *reinterpret_cast<uint32_t*>(out + (static_cast<size_t>(bs_b) * H + h) * dv + col) = pack_bf16(acc[2], acc[3]);
   }
-  TRK_END(2);
 }
 
 cudaError_t launch_combine(const transmla_params_t& p, int G, const int32_t* cum, const float* partial_o,

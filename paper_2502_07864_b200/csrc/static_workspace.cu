@@ -18,14 +18,13 @@ static __device__ __align__(256) unsigned char g_static_workspace[kStaticWorkspa
 
 // In host code `g_static_workspace` is only a handle for the runtime, not a device address, so the
 // address the kernels get is looked up once per device with that device current.
-constexpr int kMaxDevices = 64;
 std::mutex g_mutex;
-void* g_device_ptr[kMaxDevices] = {};
+void* g_device_ptr[transmla::kMaxDevices] = {};
 
 transmla_status_t static_workspace_ptr(void** out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return TRANSMLA_ERR_CUDA; }
-  if (dev < 0 || dev >= kMaxDevices) return TRANSMLA_ERR_CUDA;
+  if (dev < 0 || dev >= transmla::kMaxDevices) return TRANSMLA_ERR_CUDA;  // device ordinals beyond 63 are not served
   std::lock_guard<std::mutex> lock(g_mutex);
   if (g_device_ptr[dev] == nullptr) {
     void* p = nullptr;

@@ -168,6 +168,25 @@ def test_bad_page_index_is_reported_not_fatal():
     gu.assert_close(lifts.f64(out), want, 'bad page skipped')
 
 
+@pytest.mark.parametrize('shape', [synth.TINY, synth.LLAMA2_7B])
+def test_sequence_length_beyond_the_page_table_is_clamped_and_reported(shape):
+    # a length for which the page table has no entries: clamped to max_pages * P (nothing is read outside the
+    # table's row), reported through the status word, and the result is that of the clamped length
+    case = synth.make_decode_case(shape, [130, 192], 12)          # 3 pages per sequence, all of them owned
+    max_pages = case['page_table'].shape[1]
+    case['seqlens'][1] = max_pages * 64 + 1000
+    case['seqlens'][0] = -7
+    scale = gu.mla_scale(shape)
+    for G in (0, 3):
+        out, lse, status, _, _ = gu.gpu_decode(shape, gu.to_dev(case), scale, G=G)
+        assert status == 4
+        want_case = dict(case)
+        want_case['seqlens'] = torch.tensor([0, max_pages * 64], dtype=torch.int32)
+        want, want_lse = gu.oracle_decode(shape, want_case, scale)
+        gu.assert_close(lifts.f64(out), want, 'clamped length')
+        gu.assert_lse_close(lifts.f64(lse), want_lse, 'clamped length lse')
+
+
 def test_combine_alone_on_oracle_partials():
     # feed the oracle's per-segment partials to the CUDA combine and compare with the oracle's result
     shape = synth.TINY
