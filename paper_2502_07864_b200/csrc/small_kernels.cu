@@ -97,107 +97,115 @@ __device__ void plan_block(const int32_t* seqlens, int B, int G, int RB, int max
 
 // ------------------------------------------------------------------------------------------------
 // Absorb (Eq. 9 right, first line): q_hat[bs,h,:r] = W_UK_h^T q_nope[bs,h,:], q_hat[bs,h,r:] = q_pe[bs,h,:].
-// Block (h, rt) owns 128 latent columns of one head: it stages W_UK_h[:, tile] and the head's query
-// rows (128 at a time) in shared memory and walks the rows in 16-row tiles, so W_UK is read once.
+// A block owns nt consecutive 128-column tiles of one head's latent columns (nt = 1, or 2 when that brings the
+// launch down to one wave): it stages W_UK_h[:, tiles] and the head's query rows (128 at a time) in shared
+// memory with asynchronous 16-byte copies, all in flight together, and walks the rows in 16-row tiles, so W_UK
+// is read once.  The block that owns a head's first tile also copies the rope part of the rows.
 // ------------------------------------------------------------------------------------------------
-constexpr int kAbsorbPitch = 128 + 8;
 constexpr int kAbsorbRows = 128;  // query rows staged per pass
 
 __device__ void absorb_block(const __nv_bfloat16* q_nope, const __nv_bfloat16* q_pe,
                              const __nv_bfloat16* __restrict__ w_uk, __nv_bfloat16* q_hat, int BS, int H,
-                             int dn, int dR, int r, int h, int rt, unsigned char* smem_raw) {
-  const int apitch = dn + 8;
-  __nv_bfloat16* w_s = reinterpret_cast<__nv_bfloat16*>(smem_raw);  // [dn][kAbsorbPitch]
-  __nv_bfloat16* a_s = w_s + dn * kAbsorbPitch;                      // [kAbsorbRows][dn + 8]
+                             int dn, int dR, int r, int h, int rt0, int nt, unsigned char* smem_raw) {
+  const int apitch = dn + 8, wpitch = nt * 128 + 8;
+  __nv_bfloat16* w_s = reinterpret_cast<__nv_bfloat16*>(smem_raw);  // [dn][wpitch]
+  __nv_bfloat16* a_s = w_s + dn * wpitch;                            // [kAbsorbRows][dn + 8]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, t4 = lane & 3, mi = lane >> 3;
-  const int n0 = rt * 128, K = r + dR;
-  for (int i = tid; i < dn * 16; i += 256) {
-    const int k = i >> 4, c = i & 15;
-    uint4 v = make_uint4(0, 0, 0, 0);
-    if (n0 + c * 8 < r) v = ld_u128(w_uk + (static_cast<size_t>(h) * dn + k) * r + n0 + c * 8);
-    *reinterpret_cast<uint4*>(w_s + k * kAbsorbPitch + c * 8) = v;
+  const int n0 = rt0 * 128, K = r + dR, vec_per_row = nt * 16;
+  for (int i = tid; i < dn * vec_per_row; i += 256) {  // columns beyond r are zero-filled
+    const int k = i / vec_per_row, c = i % vec_per_row;
+    const bool in = n0 + c * 8 < r;
+    cp_async16(w_s + k * wpitch + c * 8, w_uk + (static_cast<size_t>(h) * dn + k) * r + (in ? n0 + c * 8 : 0), in ? 16 : 0);
   }
+  cp_async_commit();
   pdl_wait();  // the queries may come from the kernel before this one; the weights above may not
   const int chunks = dn / 8;
   for (int p0 = 0; p0 < BS; p0 += kAbsorbRows) {
     const int rows = min(kAbsorbRows, BS - p0);
     const int rows16 = (rows + 15) & ~15;
     if (p0 > 0) __syncthreads();  // previous pass has consumed a_s
-    if (rows16 * chunks > 256) {
-      // many rows: eight 16-byte loads per thread in flight together (one at a time costs a trip to memory each)
-      for (int i0 = tid; i0 < rows16 * chunks; i0 += 256 * 8) {
-        uint4 v[8];
+    for (int i = tid; i < rows16 * chunks; i += 256) {  // rows beyond the last one are zero-filled
+      const int rr = i / chunks, c = i % chunks;
+      cp_async16(a_s + rr * apitch + c * 8, q_nope + (static_cast<size_t>(p0 + min(rr, rows - 1)) * H + h) * dn + c * 8,
+                 rr < rows ? 16 : 0);
+    }
+    cp_async_commit();
+    if (p0 == 0 && rt0 == 0 && dR > 0) {
+      // the rope part is a plain copy, made while the operands of the first products are on their way
+      if (dR % 8 == 0 && r % 8 == 0) {  // 16 bytes at a time, four copies in flight
+        const int vecs = dR / 8;
+        for (int i0 = tid; i0 < BS * vecs; i0 += 256 * 4) {
+          uint4 v[4];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const int i = i0 + u * 256, rr = i / chunks, c = i % chunks;
-          v[u] = make_uint4(0, 0, 0, 0);
-          if (i < rows16 * chunks && rr < rows) v[u] = ld_u128(q_nope + (static_cast<size_t>(p0 + rr) * H + h) * dn + c * 8);
-        }
+          for (int u = 0; u < 4; ++u) {
+            const int i = i0 + u * 256, row = i / vecs, c = (i % vecs) * 8;
+            v[u] = make_uint4(0, 0, 0, 0);
+            if (i < BS * vecs) v[u] = ld_u128(q_pe + (static_cast<size_t>(row) * H + h) * dR + c);
+          }
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const int i = i0 + u * 256, rr = i / chunks, c = i % chunks;
-          if (i < rows16 * chunks) *reinterpret_cast<uint4*>(a_s + rr * apitch + c * 8) = v[u];
+          for (int u = 0; u < 4; ++u) {
+            const int i = i0 + u * 256, row = i / vecs, c = (i % vecs) * 8;
+            if (i < BS * vecs) *reinterpret_cast<uint4*>(q_hat + (static_cast<size_t>(row) * H + h) * K + r + c) = v[u];
+          }
         }
-      }
-    } else {
-      for (int i = tid; i < rows16 * chunks; i += 256) {
-        const int rr = i / chunks, c = i % chunks;
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (rr < rows) v = ld_u128(q_nope + (static_cast<size_t>(p0 + rr) * H + h) * dn + c * 8);
-        *reinterpret_cast<uint4*>(a_s + rr * apitch + c * 8) = v;
+      } else {
+        const int pairs = dR / 2;
+        for (int i = tid; i < BS * pairs; i += 256) {
+          const int row = i / pairs, c = (i % pairs) * 2;
+          *reinterpret_cast<uint32_t*>(q_hat + (static_cast<size_t>(row) * H + h) * K + r + c) =
+              ld_u32(q_pe + (static_cast<size_t>(row) * H + h) * dR + c);
+        }
       }
     }
+    cp_async_wait<0>();
     __syncthreads();
     for (int m0 = 0; m0 < rows16; m0 += 16) {
-      float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+      for (int wc = warp * 16 * nt; wc < (warp + 1) * 16 * nt; wc += 16) {  // this warp's 16-column steps
+        float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll 4
-      for (int ks = 0; ks < dn / 16; ++ks) {
-        uint32_t a[4], bf[4];
-        ldmatrix_x4(a, a_s + (m0 + (mi & 1) * 8 + (lane & 7)) * apitch + ks * 16 + (mi >> 1) * 8);
-        ldmatrix_x4_trans(bf, w_s + (ks * 16 + (mi & 1) * 8 + (lane & 7)) * kAbsorbPitch + warp * 16 + (mi >> 1) * 8);
-        mma_bf16_16816(acc[0], a, bf[0], bf[1]);
-        mma_bf16_16816(acc[1], a, bf[2], bf[3]);
-      }
-      const int r0 = p0 + m0 + g, r1 = r0 + 8;
+        for (int ks = 0; ks < dn / 16; ++ks) {
+          uint32_t a[4], bf[4];
+          ldmatrix_x4(a, a_s + (m0 + (mi & 1) * 8 + (lane & 7)) * apitch + ks * 16 + (mi >> 1) * 8);
+          ldmatrix_x4_trans(bf, w_s + (ks * 16 + (mi & 1) * 8 + (lane & 7)) * wpitch + wc + (mi >> 1) * 8);
+          mma_bf16_16816(acc[0], a, bf[0], bf[1]);
+          mma_bf16_16816(acc[1], a, bf[2], bf[3]);
+        }
+        const int r0 = p0 + m0 + g, r1 = r0 + 8;
 #pragma unroll
-      for (int j = 0; j < 2; ++j) {
-        const int col = n0 + warp * 16 + j * 8 + t4 * 2;
-        if (col < r) {
-          if (r0 < BS) *reinterpret_cast<uint32_t*>(q_hat + (static_cast<size_t>(r0) * H + h) * K + col) = pack_bf16(acc[j][0], acc[j][1]);
-          if (r1 < BS) *reinterpret_cast<uint32_t*>(q_hat + (static_cast<size_t>(r1) * H + h) * K + col) = pack_bf16(acc[j][2], acc[j][3]);
+        for (int j = 0; j < 2; ++j) {
+          const int col = n0 + wc + j * 8 + t4 * 2;
+          if (col < r) {
+            if (r0 < BS) *reinterpret_cast<uint32_t*>(q_hat + (static_cast<size_t>(r0) * H + h) * K + col) = pack_bf16(acc[j][0], acc[j][1]);
+            if (r1 < BS) *reinterpret_cast<uint32_t*>(q_hat + (static_cast<size_t>(r1) * H + h) * K + col) = pack_bf16(acc[j][2], acc[j][3]);
+          }
         }
       }
-    }
-  }
-  if (rt == 0 && dR > 0 && BS > 32 && dR % 8 == 0 && r % 8 == 0) {  // many rows: 16 bytes at a time, four copies in flight
-    const int vecs = dR / 8;
-    for (int i0 = tid; i0 < BS * vecs; i0 += 256 * 4) {
-      uint4 v[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int i = i0 + u * 256, row = i / vecs, c = (i % vecs) * 8;
-        v[u] = make_uint4(0, 0, 0, 0);
-        if (i < BS * vecs) v[u] = ld_u128(q_pe + (static_cast<size_t>(row) * H + h) * dR + c);
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int i = i0 + u * 256, row = i / vecs, c = (i % vecs) * 8;
-        if (i < BS * vecs) *reinterpret_cast<uint4*>(q_hat + (static_cast<size_t>(row) * H + h) * K + r + c) = v[u];
-      }
-    }
-  } else if (rt == 0 && dR > 0) {
-    const int pairs = dR / 2;
-    for (int i = tid; i < BS * pairs; i += 256) {
-      const int row = i / pairs, c = (i % pairs) * 2;
-      *reinterpret_cast<uint32_t*>(q_hat + (static_cast<size_t>(row) * H + h) * K + r + c) =
-          ld_u32(q_pe + (static_cast<size_t>(row) * H + h) * dR + c);
     }
   }
 }
 
-static size_t absorb_smem(int dn) {
-  return (static_cast<size_t>(dn) * kAbsorbPitch + static_cast<size_t>(kAbsorbRows) * (dn + 8)) * sizeof(__nv_bfloat16);
+static size_t absorb_smem(int dn, int nt) {
+  return (static_cast<size_t>(dn) * (nt * 128 + 8) + static_cast<size_t>(kAbsorbRows) * (dn + 8)) * sizeof(__nv_bfloat16);
+}
+
+// Tiles per absorb block: two when the prologue launch would otherwise not fit the device in one wave of one block
+// per SM (the append's accumulators allow no more), the tile count is even and the pair's weights fit.
+static int absorb_tiles_per_block(const transmla_params_t& p, int other_blocks) {
+  static PerDeviceFlag sms_of;  // SM count per device, asked once
+  const int slot = current_device_slot();
+  int sms = slot >= 0 ? sms_of.value[slot].load(std::memory_order_acquire) : 0;
+  if (sms == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+      cudaGetLastError();
+      return 1;
+    }
+    if (slot >= 0) sms_of.value[slot].store(sms, std::memory_order_release);
+  }
+  const int r_tiles = (p.kv_lora_rank + 127) / 128;
+  const bool fits_one = other_blocks + p.num_heads * r_tiles <= sms;
+  return (!fits_one && r_tiles % 2 == 0 && p.qk_nope_dim <= 128) ? 2 : 1;
 }
 
 __global__ void __launch_bounds__(256) append_kernel(const __nv_bfloat16* x,
@@ -224,13 +232,13 @@ __global__ void __launch_bounds__(256) absorb_plan_kernel(const __nv_bfloat16* q
                                                           __nv_bfloat16* q_hat,
                                                           const int32_t* seqlens, int32_t* cum,
                                                           int32_t* plan, int32_t* dev_status, int B, int S, int H,
-                                                          int dn, int dR, int r, int G, int max_pages) {
+                                                          int dn, int dR, int r, int G, int max_pages, int nt) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   pdl_trigger();
-  const int r_tiles = (r + 127) / 128;
-  const int n_absorb = H * r_tiles;
+  const int per_head = (r + 127) / 128 / nt;  // absorb blocks per head, nt tiles each
+  const int n_absorb = H * per_head;
   if (static_cast<int>(blockIdx.x) < n_absorb) {
-    absorb_block(q_nope, q_pe, w_uk, q_hat, B * S, H, dn, dR, r, blockIdx.x / r_tiles, blockIdx.x % r_tiles, smem_raw);
+    absorb_block(q_nope, q_pe, w_uk, q_hat, B * S, H, dn, dR, r, blockIdx.x / per_head, blockIdx.x % per_head * nt, nt, smem_raw);
   } else {
     plan_block(seqlens, B, G, (S * H + kRowBlock - 1) / kRowBlock, max_pages, cum, plan, dev_status, smem_raw);
   }
@@ -243,11 +251,11 @@ __global__ void __launch_bounds__(256) prologue_kernel(
     const int32_t* page_table, __nv_bfloat16* cache, const __nv_bfloat16* q_nope,
     const __nv_bfloat16* q_pe, const __nv_bfloat16* __restrict__ w_uk, __nv_bfloat16* q_hat,
     const int32_t* seqlens, int32_t* cum, int32_t* plan, int32_t* dev_status, int B, int S, int H, int D,
-    int dn, int dR, int r, int num_pages, int max_pages, float theta, int G, int t_splits, int wide) {
+    int dn, int dR, int r, int num_pages, int max_pages, float theta, int G, int t_splits, int wide, int nt) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   pdl_trigger();
   const int n_append = (r + dR) / (wide ? 32 : 8) * t_splits;
-  const int r_tiles = (r + 127) / 128;
+  const int per_head = (r + 127) / 128 / nt;  // absorb blocks per head, nt tiles each
   const int bid = static_cast<int>(blockIdx.x) - 1;
   if (bid < 0) {
     plan_block(seqlens, B, G, (S * H + kRowBlock - 1) / kRowBlock, max_pages, cum, plan, dev_status, smem_raw);
@@ -260,7 +268,7 @@ __global__ void __launch_bounds__(256) prologue_kernel(
                                     max_pages, theta, bid, t_splits, smem_raw);
   } else {
     const int a = bid - n_append;
-    absorb_block(q_nope, q_pe, w_uk, q_hat, B * S, H, dn, dR, r, a / r_tiles, a % r_tiles, smem_raw);
+    absorb_block(q_nope, q_pe, w_uk, q_hat, B * S, H, dn, dR, r, a / per_head, a % per_head * nt, nt, smem_raw);
   }
 }
 
@@ -293,14 +301,15 @@ cudaError_t launch_absorb_plan(const transmla_params_t& p, int G, const __nv_bfl
                                const __nv_bfloat16* q_pe, const __nv_bfloat16* w_uk, __nv_bfloat16* q_hat,
                                const int32_t* seqlens, int32_t* cum, int32_t* plan, int32_t* dev_status,
                                cudaStream_t stream) {
-  size_t smem = absorb_smem(p.qk_nope_dim);
+  const int nt = absorb_tiles_per_block(p, 1);
+  size_t smem = absorb_smem(p.qk_nope_dim, nt);
   if (smem < kPlanSmemSeqs * sizeof(int32_t)) smem = kPlanSmemSeqs * sizeof(int32_t);
   static PerDeviceFlag smem_set;  // zero-initialised; one slot per device
   if (cudaError_t e = ensure_dynamic_smem(absorb_plan_kernel, kPrologueMaxSmem, smem_set); e != cudaSuccess) return e;
-  const int blocks = p.num_heads * ((p.kv_lora_rank + 127) / 128) + 1;
+  const int blocks = p.num_heads * ((p.kv_lora_rank + 127) / 128 / nt) + 1;
   return launch_pdl(absorb_plan_kernel, dim3(blocks), dim3(256), smem, stream, q_nope, q_pe, w_uk, q_hat, seqlens, cum,
                     plan, dev_status, p.batch, p.q_len, p.num_heads, p.qk_nope_dim, p.qk_rope_dim, p.kv_lora_rank, G,
-                    p.max_pages_per_seq);
+                    p.max_pages_per_seq, nt);
 }
 
 cudaError_t launch_prologue(const transmla_params_t& p, int G, const __nv_bfloat16* x, const __nv_bfloat16* w_dkv_kr,
@@ -308,16 +317,18 @@ cudaError_t launch_prologue(const transmla_params_t& p, int G, const __nv_bfloat
                             const __nv_bfloat16* q_pe, const __nv_bfloat16* w_uk, __nv_bfloat16* q_hat,
                             const int32_t* seqlens, int32_t* cum, int32_t* plan, int32_t* dev_status,
                             cudaStream_t stream) {
-  size_t smem = absorb_smem(p.qk_nope_dim);
+  const int ts = append_token_splits(p);
+  const int wide = append_wide(p) ? 1 : 0;
+  const int n_append = (p.kv_lora_rank + p.qk_rope_dim) / (wide ? 32 : 8) * ts;
+  const int nt = absorb_tiles_per_block(p, 1 + n_append);
+  size_t smem = absorb_smem(p.qk_nope_dim, nt);
   if (smem < kAppendSmem) smem = kAppendSmem;
   static PerDeviceFlag smem_set;  // zero-initialised; one slot per device
   if (cudaError_t e = ensure_dynamic_smem(prologue_kernel, kPrologueMaxSmem, smem_set); e != cudaSuccess) return e;
-  const int ts = append_token_splits(p);
-  const int wide = append_wide(p) ? 1 : 0;
-  const int blocks = 1 + (p.kv_lora_rank + p.qk_rope_dim) / (wide ? 32 : 8) * ts + p.num_heads * ((p.kv_lora_rank + 127) / 128);
+  const int blocks = 1 + n_append + p.num_heads * ((p.kv_lora_rank + 127) / 128 / nt);
   return launch_pdl(prologue_kernel, dim3(blocks), dim3(256), smem, stream, x, w_dkv_kr, page_table, cache, q_nope, q_pe,
                     w_uk, q_hat, seqlens, cum, plan, dev_status, p.batch, p.q_len, p.num_heads, p.hidden_dim,
-                    p.qk_nope_dim, p.qk_rope_dim, p.kv_lora_rank, p.num_pages, p.max_pages_per_seq, p.rope_theta, G, ts, wide);
+                    p.qk_nope_dim, p.qk_rope_dim, p.kv_lora_rank, p.num_pages, p.max_pages_per_seq, p.rope_theta, G, ts, wide, nt);
 }
 
 // ------------------------------------------------------------------------------------------------
