@@ -173,10 +173,37 @@ def run_reference(args, name, shape, seqlens, seed):
     }))
 
 
+def kernel_source_hash():
+    """Hash of the sources the split-KV kernel is compiled from; ties an ncu capture to the code it was taken on."""
+    import hashlib
+    h = hashlib.sha256()
+    for f in ('decode_sm100.cu', 'common.cuh', 'sm100_ptx.cuh'):
+        h.update(open(os.path.join(ROOT, 'paper_2502_07864_b200', 'csrc', f), 'rb').read())
+    return h.hexdigest()[:16]
+
+
+def traffic_from_profile(name):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one split-KV launch, from the ncu summary under profiles/ for
+    this workload; None when there is none or when the kernel's sources have changed since the capture."""
+    path = os.path.join(ROOT, 'profiles', f'decode_sm100_{name.replace("-mla", "")}.md')
+    try:
+        text = open(path).read()
+    except OSError:
+        return None
+    vals = {}
+    for line in text.splitlines():
+        if line.startswith('traffic_bytes_per_launch:') or line.startswith('kernel_source_hash:'):
+            k, v = line.split(':', 1)
+            vals[k] = v.strip()
+    if vals.get('kernel_source_hash') != kernel_source_hash() or 'traffic_bytes_per_launch' not in vals:
+        return None
+    return float(vals['traffic_bytes_per_launch'])
+
+
 def run_ours(args, name, shape, seqlens, seed):
     import torch
     import torch.distributed as dist
-    from paper_2502_07864_b200 import binding, build, replicas, synth
+    from paper_2502_07864_b200 import binding, build, replicas
 
     rank = int(os.environ.get('RANK', '0'))
     world = int(os.environ.get('WORLD_SIZE', '1'))
@@ -190,6 +217,31 @@ def run_ours(args, name, shape, seqlens, seed):
         dist.barrier()
     binding.lib()          # raises if the CUDA library is missing: there is no other path
 
+    line = measure(args, name, shape, seqlens, seed, rank, world, local, full=True)
+    if rank == 0:
+        if world == 1 and args.sweep:
+            # the other rows of the target range, each measured the same way (shorter), so that one run shows them all
+            line['sweep'] = []
+            for other in args.sweep.split(','):
+                if other and other != name:
+                    sh, sl, sd = workloads()[other]
+                    row = measure(args, other, sh, sl, sd, rank, world, local, full=False)
+                    line['sweep'].append({k: row[k] for k in ('config', 'ms_per_step', 'value', 'decode_kernel_us',
+                                                               'cache_gbs_pct_of_8tbs', 'roofline', 'clocks')})
+        if world == 1 and not args.no_cpu_baseline:
+            line['cpu_baseline'] = cpu_baseline(shape, seqlens, seed, (shape.dn + shape.dR) ** -0.5)
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def measure(args, name, shape, seqlens, seed, rank, world, local, full):
+    """One workload: whole-step time over args.steps steps, split-KV kernel time, read-probe ceiling, and (full) the
+    host-buffer end-to-end figure and the optional layer step.  Returns the JSON line as a dict (rank 0)."""
+    import torch
+    from paper_2502_07864_b200 import binding, replicas, synth
+
+    steps = args.steps if full else min(args.steps, 200)
     B, S, H = len(seqlens), shape.S, shape.H
     scale = (shape.dn + shape.dR) ** -0.5
     n_copies = args.cache_copies
@@ -225,7 +277,7 @@ def run_ours(args, name, shape, seqlens, seed):
 
     # The split-KV kernel is timed by events the library records around it, on every 8th step of the timed
     # region only: an event record between two kernels switches off their launch overlap for that step.
-    sampled = list(range(0, args.steps, 8))
+    sampled = list(range(0, steps, 8))
     kev = {i: (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for i in sampled}
     for a, b_ in kev.values():       # create the underlying CUDA events before handing them to the library
         a.record(stream); b_.record(stream)
@@ -234,43 +286,72 @@ def run_ours(args, name, shape, seqlens, seed):
     barrier()
     t0 = time.perf_counter()
     e0.record(stream)
-    for i in range(args.steps):
+    for i in range(steps):
         step(i, kev.get(i))
     e1.record(stream)
     barrier()
     t1 = time.perf_counter()
     ms_total = e0.elapsed_time(e1)
     clocks = sampler.stop(t0, t1) if sampler else None
-    kernel_ms = statistics.mean(a.elapsed_time(b_) for a, b_ in kev.values())
+    kernel_times = [a.elapsed_time(b_) for a, b_ in kev.values()]
+    # At least 16 launches of the split-KV kernel are timed whatever --steps is: what the timed region did not give
+    # comes from extra steps after it, each with the library's events around its split-KV kernel.
+    extra = max(0, 16 - len(kernel_times))
+    for i in range(extra):
+        ev = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+        ev[0].record(stream); ev[1].record(stream)
+        step(steps + i, ev)
+        torch.cuda.synchronize()
+        kernel_times.append(ev[0].elapsed_time(ev[1]))
+    kernel_ms = statistics.mean(kernel_times)
     word = int(status.item())
     assert word == 0, f'device status word {word:#x} after the timed steps'
 
-    # end to end through the host-buffer entry point: pinned host inputs, result read back every step
-    staging = torch.empty(binding.transmla_step_staging_bytes(params), dtype=torch.uint8, device='cuda')
-    pin = lambda t: t.cpu().contiguous().pin_memory()
-    h = {k: pin(v) for k, v in (('x', ac['x']), ('q_nope', dc['q_nope']), ('q_pe', dc['q_pe']),
-                                ('page_table', dc['page_table']), ('seqlens', dc['seqlens']))}
-    h_out = torch.empty(B, S, H, shape.dv, dtype=torch.bfloat16).pin_memory()
-    h_lse = torch.empty(B, S, H, dtype=torch.float32).pin_memory()
+    # Read-only streaming probe: the same pages through the same grid and TMA ring with nothing computed; its time is
+    # the floor under the split-KV kernel for this workload (r = 512, dR = 64 only).
+    probe_us = None
+    if shape.r == 512 and shape.dR == 64:
+        probe = []
+        for i in range(3 + 20):
+            ev = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+            ev[0].record(stream)
+            binding.transmla_stream_probe(params, caches[i % n_copies], dc['page_table'], ws, status, stream)
+            ev[1].record(stream)
+            torch.cuda.synchronize()
+            if i >= 3:
+                probe.append(ev[0].elapsed_time(ev[1]) * 1e3)
+        probe_us = statistics.median(probe)
 
-    def host_step(i):
-        word = binding.transmla_decode_step_host(params, h['x'], h['q_nope'], h['q_pe'], h['page_table'], h['seqlens'],
-                                                 *weights[i % n_w], caches[i % n_copies], staging,
-                                                 ws, h_out, h_lse, stream)
-        assert word == 0, f'device status word {word:#x} in host step {i}'
-    for i in range(3):
-        host_step(i)
-    barrier()
-    t2 = time.perf_counter()
-    for i in range(args.steps):
-        host_step(i)
-    barrier()
-    e2e_s = time.perf_counter() - t2
-    h2d = sum(v.numel() * v.element_size() for v in h.values())
-    d2h = h_out.numel() * 2 + h_lse.numel() * 4 + 4
+    # end to end through the host-buffer entry point: pinned host inputs, result read back every step
+    def end_to_end():
+        staging = torch.empty(binding.transmla_step_staging_bytes(params), dtype=torch.uint8, device='cuda')
+        pin = lambda t: t.cpu().contiguous().pin_memory()
+        h = {k: pin(v) for k, v in (('x', ac['x']), ('q_nope', dc['q_nope']), ('q_pe', dc['q_pe']),
+                                    ('page_table', dc['page_table']), ('seqlens', dc['seqlens']))}
+        h_out = torch.empty(B, S, H, shape.dv, dtype=torch.bfloat16).pin_memory()
+        h_lse = torch.empty(B, S, H, dtype=torch.float32).pin_memory()
+
+        def host_step(i):
+            word = binding.transmla_decode_step_host(params, h['x'], h['q_nope'], h['q_pe'], h['page_table'], h['seqlens'],
+                                                     *weights[i % n_w], caches[i % n_copies], staging,
+                                                     ws, h_out, h_lse, stream)
+            assert word == 0, f'device status word {word:#x} in host step {i}'
+        for i in range(3):
+            host_step(i)
+        barrier()
+        t2 = time.perf_counter()
+        for i in range(steps):
+            host_step(i)
+        barrier()
+        e2e_s = time.perf_counter() - t2
+        h2d = sum(v.numel() * v.element_size() for v in h.values())
+        d2h = h_out.numel() * 2 + h_lse.numel() * 4 + 4
+        return e2e_s, h2d, d2h
+
+    e2e_s, h2d, d2h = end_to_end() if full else (float('nan'), 0, 0)   # skipped for the rows of the sweep
 
     layer = None
-    if args.layer:
+    if args.layer and full:
         # the whole attention layer (queries -> the step above -> W_O) on device buffers; its weights rotate too
         lws = []
         for i in range(args.layer_weight_copies):
@@ -288,13 +369,13 @@ def run_ours(args, name, shape, seqlens, seed):
         barrier()
         l0, l1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         l0.record(stream)
-        for i in range(args.steps):
+        for i in range(steps):
             layer_step(i)
         l1.record(stream)
         barrier()
         word = int(status.item())
         assert word == 0, f'device status word {word:#x} after the layer steps'
-        layer_ms = replicas.max_over_ranks([l0.elapsed_time(l1)], device='cuda')[0] / args.steps
+        layer_ms = replicas.max_over_ranks([l0.elapsed_time(l1)], device='cuda')[0] / steps
         lbytes = sum(t.numel() * t.element_size() for t in lws[0].values())
         layer = {'ms_per_step': layer_ms, 'tokens_per_s': B * S * world / (layer_ms * 1e-3), 'weight_bytes': lbytes,
                  'q_lora_rank': args.q_lora_rank, 'launches_per_step': 6 + (1 if args.q_lora_rank else 0),
@@ -302,12 +383,10 @@ def run_ours(args, name, shape, seqlens, seed):
 
     ms_total, e2e_ms = replicas.max_over_ranks([ms_total, e2e_s * 1e3], device='cuda')
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return
+        return None
 
     tokens_per_step = B * S * world
-    ms_step = ms_total / args.steps
+    ms_step = ms_total / steps
     cache_bytes = sum(seqlens) * shape.row * 2                       # live latent rows, read once
     q_hat_bytes = B * S * H * shape.row * 2
     algo_bytes = cache_bytes + q_hat_bytes                           # per split-KV launch
@@ -317,39 +396,41 @@ def run_ours(args, name, shape, seqlens, seed):
     flops = 2.0 * (shape.row + shape.r) * H * S * sum(seqlens)
     tpeak, tpeak_kind = measured_tensor_peak()
     tflops = flops / (kernel_ms * 1e-3) / 1e12
-    # ncu dram__bytes_read.sum + dram__bytes_write.sum of one split-KV launch on the default workload
-    # (profiles/decode_sm100_llama2-7b_b16_8k.md); other workloads have no capture
-    traffic = 155.63e6 if name == 'llama2-7b-mla_b16_8k' and world == 1 else None
+    # ncu dram__bytes_read.sum + dram__bytes_write.sum of one split-KV launch of this workload, as recorded in the
+    # summary under profiles/ together with a hash of the kernel's sources; null once those have changed
+    traffic = traffic_from_profile(name) if world == 1 else None
+    claims = 'run-time' if binding.transmla_page_claims_at_run_time(params) else 'planned'
     line = {
-        'metric': METRIC, 'value': replicas.whole_job_rate(B * S, args.steps, ms_total), 'unit': 'tokens/s', 'n_gpus': world,
-        'steps': args.steps, 'warmup': max(args.warmup, 3), 'ms_per_step': ms_step, 'higher_is_better': True,
+        'metric': METRIC, 'value': replicas.whole_job_rate(B * S, steps, ms_total), 'unit': 'tokens/s', 'n_gpus': world,
+        'steps': steps, 'warmup': max(args.warmup, 3), 'ms_per_step': ms_step, 'higher_is_better': True,
         'scaling': 'weak', 'vs_baseline': None, 'dtype': 'bf16', 'data': 'synthetic',
         'config': {'workload': name, 'batch_per_gpu': B, 'q_len': S, 'heads': H, 'latent': shape.r, 'rope': shape.dR,
                    'cached_tokens_per_gpu': sum(seqlens), 'page_size': shape.page_size,
-                   'num_partitions': lay.num_partitions,
+                   'num_partitions': lay.num_partitions, 'page_claims': claims,
                    'l2': f'cache rotates over {n_copies} copies ({n_copies * cache_bytes / 1e6:.0f} MB) and the weights '
                          f'over {n_w} copies ({n_w * weight_bytes / 1e6:.0f} MB) between steps',
                    'parallelism': f'replicas x{world}, no data-path collective'},
         'cache_gbs': world * cache_bytes / (ms_step * 1e-3) / 1e9,
         'cache_gbs_pct_of_8tbs': 100.0 * cache_bytes / (ms_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
-        'decode_kernel_us': kernel_ms * 1e3, 'decode_kernel_launches_timed': len(kev),
+        'decode_kernel_us': kernel_ms * 1e3, 'decode_kernel_launches_timed': len(kernel_times),
+        'decode_kernel_timing': f'library events around the split-KV kernel: every 8th step of the timed region ({len(kev)}) '
+                                f'and {extra} extra steps after it',
         'roofline': {'bound': 'hbm', 'achieved': achieved, 'peak': peak, 'unit': 'GB/s', 'frac': achieved / peak,
                      'peak_kind': f'{peak_kind} copy bandwidth', 'frac_of_8tbs': achieved / NOMINAL_HBM_GBS,
                      'kernel': 'split-KV decode', 'algorithmic_bytes_per_launch': algo_bytes, 'traffic': traffic,
+                     'traffic_source': 'ncu capture summarised under profiles/ (null: none for this workload, or the kernel changed since)',
+                     'read_probe_us': probe_us,
+                     'read_probe_gbs': None if probe_us is None else cache_bytes / probe_us / 1e3,
                      'tensor': {'achieved_tflops': tflops, 'peak_tflops': tpeak, 'peak_kind': f'{tpeak_kind} bf16 GEMM',
                                 'frac': tflops / tpeak, 'flops_per_launch': flops}},
-        'e2e': {'value': replicas.whole_job_rate(B * S, args.steps, e2e_ms), 'unit': 'tokens/s',
-                'h2d_bytes_per_step': h2d, 'd2h_bytes_per_step': d2h, 'ms_per_step': e2e_ms / args.steps},
-        'gpu_launches': KERNELS_PER_STEP * args.steps,
+        'e2e': {'value': replicas.whole_job_rate(B * S, steps, e2e_ms), 'unit': 'tokens/s',
+                'h2d_bytes_per_step': h2d, 'd2h_bytes_per_step': d2h, 'ms_per_step': e2e_ms / steps},
+        'gpu_launches': KERNELS_PER_STEP * steps,
         'clocks': clocks,
     }
     if layer is not None:
         line['layer'] = layer
-    if world == 1 and not args.no_cpu_baseline:
-        line['cpu_baseline'] = cpu_baseline(shape, seqlens, seed, scale)
-    print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    return line
 
 
 def main():
@@ -365,6 +446,8 @@ def main():
     ap.add_argument('--layer', action='store_true', help='also time the whole layer step (queries, attention, W_O)')
     ap.add_argument('--q-lora-rank', type=int, default=0, help='low-rank queries for --layer (0: full rank)')
     ap.add_argument('--layer-weight-copies', type=int, default=6)
+    ap.add_argument('--sweep', default='llama2-7b-mla_b64_8k,llama2-7b-mla_b128_8k,qwen2.5-72b-mla_b64_s2',
+                    help='comma-separated workloads measured after the main one (1 GPU; empty: none)')
     args = ap.parse_args()
     w = workloads()
     if args.workload not in w:

@@ -291,6 +291,13 @@ transmla_status_t transmla_mla_attention_static(const transmla_params_t* params 
  * usable.  cycles_out (device int64[2], may be NULL) receives the SM cycles spent in the two waits. */
 transmla_status_t transmla_selftest_bounded_wait(int32_t* dev_status, long long* cycles_out, void* stream);
 
+/* Whether transmla_mla_decode with these `params` hands pages to CTAs at run time (1) or keeps to the page ranges of
+ * the split plan (0); see transmla_params_t.num_partitions.  With run-time claims the default path is not
+ * bit-stable from run to run (results agree to fp32 rounding); pass the partition count that
+ * transmla_workspace_layout reports as an explicit num_partitions to get the planned, bit-stable path.  (No
+ * counterpart in the paper: the split is this library's own.) */
+int transmla_page_claims_at_run_time(const transmla_params_t* params /* host */);
+
 /* Diagnostic: read-only streaming probe (no counterpart in the paper; it measures, it computes nothing).  Streams
  * exactly the pages that the split-KV kernel of transmla_mla_decode reads for `params` - same grid, same split
  * plan (taken from the workspace that a preceding transmla_mla_decode with the same `params` filled), same ring of

@@ -15,7 +15,7 @@ EXPORTS = ('transmla_workspace_layout', 'transmla_latent_append', 'transmla_mla_
            'transmla_validate_tables', 'transmla_step_staging_bytes', 'transmla_decode_step_host',
            'transmla_decode_step', 'transmla_profile_decode_kernel', 'transmla_status_string',
            'transmla_static_workspace_capacity', 'transmla_mla_attention_static', 'transmla_selftest_bounded_wait',
-           'transmla_layer_scratch_bytes', 'transmla_layer_decode_step', 'transmla_stream_probe')
+           'transmla_layer_scratch_bytes', 'transmla_layer_decode_step', 'transmla_stream_probe', 'transmla_page_claims_at_run_time')
 
 
 class Params(ctypes.Structure):
@@ -73,6 +73,7 @@ def lib():
         L.transmla_mla_attention_static.argtypes = [pp, vp, vp, vp, vp, vp, i32p, i32p, vp, vp, i32p, vp]
         L.transmla_selftest_bounded_wait.argtypes = [i32p, vp, vp]
         L.transmla_stream_probe.argtypes = [pp, vp, i32p, vp, sz, i32p, vp]
+        L.transmla_page_claims_at_run_time.argtypes = [pp]
         L.transmla_layer_scratch_bytes.argtypes = [pp, ctypes.c_int32]
         L.transmla_layer_scratch_bytes.restype = sz
         L.transmla_layer_decode_step.argtypes = [pp, ctypes.POINTER(LayerWeights), vp, i32p, i32p, vp, vp, sz, vp, sz, vp,
@@ -206,6 +207,10 @@ def transmla_layer_decode_step(params, weights, x, page_table, seqlens, cache, w
 def transmla_selftest_bounded_wait(dev_status, cycles_out=None, stream=None):
     _check(lib().transmla_selftest_bounded_wait(_ptr(dev_status), _ptr(cycles_out), _stream(stream)),
            'transmla_selftest_bounded_wait')
+
+
+def transmla_page_claims_at_run_time(params):
+    return bool(lib().transmla_page_claims_at_run_time(ctypes.byref(params)))
 
 
 def transmla_stream_probe(params, cache, page_table, workspace, dev_status=None, stream=None):

@@ -240,6 +240,12 @@ transmla_status_t transmla_mla_combine(const transmla_params_t* p, const void* w
   return e == cudaSuccess ? TRANSMLA_OK : TRANSMLA_ERR_CUDA;
 }
 
+int transmla_page_claims_at_run_time(const transmla_params_t* p) {
+  transmla_workspace_layout_t lay;
+  if (transmla_workspace_layout(p, &lay) != TRANSMLA_OK) return 0;
+  return dynamic_claims(*p, lay.num_partitions) ? 1 : 0;
+}
+
 transmla_status_t transmla_stream_probe(const transmla_params_t* p, const void* cache, const int32_t* page_table,
                                         const void* workspace, size_t workspace_bytes, int32_t* dev_status,
                                         void* stream) {
