@@ -15,7 +15,9 @@
 //
 // Warp roles: warps 0-3 softmax + epilogue (warp w owns tensor-memory lanes 32w..32w+31, i.e. replica w
 // of the 32 query rows, and the probabilities of tokens 16w..16w+15 of every page); warp 4 lane 0
-// issues TMA; warp 5 issues MMA (warp-uniform control flow, one elected lane per instruction).  All waits are bounded: on expiry the CTA raises
+// issues TMA; warp 5 issues the QK^T instructions and warp 6 the PV instructions (warp-uniform control flow, one
+// elected lane per instruction; two warps because issuing costs a warp about 45 cycles per instruction, more than
+// the 20 to 36 cycles these small instructions occupy the pipe).  All waits are bounded: on expiry the CTA raises
 // TRANSMLA_DEV_TIMEOUT, every later wait returns at once, and control flow stays identical, so the CTA
 // still reaches its teardown and frees its tensor memory.
 #include "common.cuh"
@@ -31,7 +33,7 @@ constexpr int kStageBytes = kChunks * kSubTileBytes;  // 73728
 constexpr int kStages = 3;
 constexpr int kPBytes = kRowBlock * 128;              // 4096: P[32 rows][64 tokens] bf16
 constexpr int kQTileBytes = kRowBlock * 128;          // 4096: one 64-column sub-tile of the 32 query rows
-constexpr int kThreads = 192;
+constexpr int kThreads = 224;
 constexpr uint32_t kTmemCols = 512;
 constexpr int kMetaRing = 16;            // descriptions of the ring items in flight (a power of two >= 2 * kStages)
 enum { ITEM_QUERIES = 1, ITEM_PAGE = 2, ITEM_END = 3 };
@@ -213,45 +215,19 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
         __syncwarp();
       }
     } else if (warp == 5) {
-      // ======================================================================== MMA issuer
+      // ======================================================================== MMA issuer, scores
       // Follows the ring: skips query items (the softmax warps move them to tensor memory and report through
-      // Q_READY, which also tells when the ring has ended), runs QK^T for a page as soon as it has landed and
-      // the PV of the page before it one step later.
+      // Q_READY, which also tells when the ring has ended) and runs QK^T for a page as soon as it has landed.
+      // Issuing an instruction costs this warp about as many cycles as a small one occupies the pipe, so the 36
+      // score instructions and the 16 product instructions of a page are issued by two warps side by side.
       constexpr uint32_t idesc_qk = instr_desc(kPage, false);
-      constexpr uint32_t idesc_pv = instr_desc(kRowBlock, true);
       int g = 0, n = 0, seg = 0;  // ring items, pages, segments handled so far
-      auto issue_pv = [&](int gr, int gp, bool first_of_segment) {  // O^T += C^T P^T for page gp held in ring item gr
-        const int stage = gr % kStages;
-        // One barrier per P buffer: the softmax warps can run a page ahead of this warp (S is ready before the PV
-        // of the page before it is issued), and with a single barrier two of its phases could complete before this
-        // wait looks at the first.  Per buffer the next phase needs the PV issued below to have completed.
-        mbar_wait(bar(BAR_P_READY0 + (gp & 1)), (gp >> 1) & 1, abort_flag, dev_status);
-        tc_fence_after();
-        const uint64_t a0 = smem_desc(base + kOffStage + stage * kStageBytes, kSubTileBytes, 1024);
-        const uint64_t b0 = smem_desc(base + kOffP + (gp & 1) * kPBytes, 16, 1024);
-        const uint32_t acc0 = first_of_segment ? 0u : 1u;
-#pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
-#pragma unroll
-          for (int t = 0; t < 4; ++t) {
-            if (elect_one())
-              mma_ss(tmem + kColO + t * 32, desc_advance(a0, (2 * t) * kSubTileBytes + kk * 2048),
-                     desc_advance(b0, kk * 32), idesc_pv, kk == 0 ? acc0 : 1u);
-          }
-        }
-        if (elect_one()) {
-          tc_commit(bar(BAR_KV_EMPTY + stage));
-          tc_commit(bar(BAR_PV_DONE0 + (gp & 1)));
-        }
-        __syncwarp();
-      };
       while (true) {
         // a segment begins (or the ring ends): the softmax warps say which
         mbar_wait(bar(BAR_Q_READY), seg & 1, abort_flag, dev_status);
         ++seg;
         if (__any_sync(0xffffffffu, *abort_flag != 0) || *ring_done != 0) break;
         ++g;  // the query item
-        bool pending = false, pending_first = false;
         while (true) {
           const int stage = g % kStages, use = g / kStages;
           mbar_wait(bar(BAR_KV_FULL + stage), use & 1, abort_flag, dev_status);
@@ -270,15 +246,53 @@ decode_sm100_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_
           }
           if (elect_one()) tc_commit(bar(BAR_S_FULL));
           __syncwarp();
-          if (pending) issue_pv(g - 1, n - 1, pending_first);
-          pending = true;
-          pending_first = (m.w & 1) != 0;
           ++g; ++n;
           if ((m.w & 2) != 0 || m.x != ITEM_PAGE || __any_sync(0xffffffffu, *abort_flag != 0)) break;
         }
-        issue_pv(g - 1, n - 1, pending_first);
       }
-    } else {
+    } else if (warp == 6) {
+      // ======================================================================== MMA issuer, products
+      // Follows the ring in the same way and issues O^T += C^T P^T for a page as soon as its probabilities are
+      // there; its commit hands the page's stage back to the TMA warp (the scores of the page are complete by
+      // then: the probabilities were made from them).
+      constexpr uint32_t idesc_pv = instr_desc(kRowBlock, true);
+      int g = 0, n = 0, seg = 0;
+      while (true) {
+        mbar_wait(bar(BAR_Q_READY), seg & 1, abort_flag, dev_status);
+        ++seg;
+        if (__any_sync(0xffffffffu, *abort_flag != 0) || *ring_done != 0) break;
+        ++g;
+        while (true) {
+          const int stage = g % kStages, use = g / kStages;
+          mbar_wait(bar(BAR_KV_FULL + stage), use & 1, abort_flag, dev_status);
+          const int4 m = meta[g & (kMetaRing - 1)];
+          // One barrier per P buffer: the softmax warps can deliver P(n) and P(n+1) back to back, and with a single
+          // barrier two of its phases could complete before this wait looks at the first.  Per buffer the next
+          // phase needs the PV issued below to have completed.
+          mbar_wait(bar(BAR_P_READY0 + (n & 1)), (n >> 1) & 1, abort_flag, dev_status);
+          tc_fence_after();
+          const uint64_t a0 = smem_desc(base + kOffStage + stage * kStageBytes, kSubTileBytes, 1024);
+          const uint64_t b0 = smem_desc(base + kOffP + (n & 1) * kPBytes, 16, 1024);
+          const uint32_t acc0 = (m.w & 1) != 0 ? 0u : 1u;  // the segment's first page starts the accumulator afresh
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk) {
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+              if (elect_one())
+                mma_ss(tmem + kColO + t * 32, desc_advance(a0, (2 * t) * kSubTileBytes + kk * 2048),
+                       desc_advance(b0, kk * 32), idesc_pv, kk == 0 ? acc0 : 1u);
+            }
+          }
+          if (elect_one()) {
+            tc_commit(bar(BAR_KV_EMPTY + stage));
+            tc_commit(bar(BAR_PV_DONE0 + (n & 1)));
+          }
+          __syncwarp();
+          ++g; ++n;
+          if ((m.w & 2) != 0 || m.x != ITEM_PAGE || __any_sync(0xffffffffu, *abort_flag != 0)) break;
+        }
+      }
+    } else if (warp < 4) {
       // ======================================================================== softmax + epilogue (warps 0-3)
       const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
       const int my_row = rb * kRowBlock + lane;  // query row of this thread (same in all four replicas)
