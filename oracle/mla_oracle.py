@@ -20,9 +20,15 @@ itself pinned to torch's scaled_dot_product_attention (Sec. 4.1, App. A.2.1), or
 re-basing of the latent (App. D.2), key/value balancing (Eq. 19), page-permutation invariance,
 partition invariance of split + combine, brute-force restatement of the split plan.
 
+FP8 latent cache (end of the file): the e4m3 format is pinned to the values of its published
+definition and to torch's float8_e4m3fn conversions, the quantiser to its error bound and to exact
+round trips of representable rows, the attention over an FP8 cache to Eq. 9 over the dequantised rows
+(tests/test_oracle_fp8.py).
+
 Parity unpinned (no statement in the paper to pin against; fixed by this library's own
 definition): the causal reading for S > 1 (query s sees tokens [0, L_b - S + s]), the result for
-L_b = 0 (zeros and lse = -inf), and that page tails are ignored.
+L_b = 0 (zeros and lse = -inf), that page tails are ignored, and the stored format of the FP8 cache
+(per-token scale, e4m3 codes of c / scale, k^R / scale in bf16): the paper only names FP8.
 """
 import numpy as np
 
@@ -336,3 +342,91 @@ def mla_layer_decode(x, w_uq, w_qr, w_dkv_kr, w_uk, w_uv, w_o, cache, page_table
     o, _ = mla_decode_mha_form(q_nope.reshape(B, S, H, -1), q_pe.reshape(B, S, H, -1), w_uk, w_uv, cache, page_table,
                                seqlens, scale, page_size)
     return output_projection(o, w_o)
+
+
+# --------------------------------------------------------------------------------------------
+# FP8 latent cache (the paper's abstract names FP8 quantisation as combinable with the method and says no more;
+# the stored format below is this library's own reading).
+#
+# A cache row of one token holds, instead of r + dR bf16 values:
+#   codes  r bytes   e4m3 codes of c_t / scale_t
+#   k_pe   dR bf16   k^R_t / scale_t, rounded to bf16   (stored pre-divided so that a score is scale_t times one sum)
+#   scale  1 fp32    scale_t = max_i |c_t[i]| / 448, rounded to fp32 (1.0 for an all-zero row)
+# The value the attention sees is the dequantised row: c~_t = scale_t * decode(codes), k~R_t = scale_t * k_pe, and the
+# result is Eq. 9 (MHA form above) on those values.  e4m3 is the 8-bit format of the OCP 8-bit floating point
+# specification: 1 sign, 4 exponent (bias 7), 3 mantissa bits, no infinities, S.1111.111 = NaN, largest finite 448.
+# --------------------------------------------------------------------------------------------
+E4M3_MAX = 448.0
+
+
+def e4m3_decode(codes):
+    """Value of each e4m3 code (uint8 array) as float64; the two NaN codes decode to NaN."""
+    codes = np.asarray(codes, dtype=np.uint8)
+    sign = np.where(codes & 0x80, -1.0, 1.0)
+    e = ((codes >> 3) & 0xF).astype(np.int64)
+    m = (codes & 0x7).astype(np.float64)
+    normal = sign * np.exp2(e - 7.0) * (1.0 + m / 8.0)
+    subnormal = sign * np.exp2(-6.0) * (m / 8.0)
+    out = np.where(e == 0, subnormal, normal)
+    return np.where((codes & 0x7F) == 0x7F, np.nan, out)
+
+
+def e4m3_encode(x):
+    """Nearest e4m3 code of each value (ties to the even code), saturating at +-448.  Written as a search over the
+    126 non-negative finite codes, so that it shares nothing with the decoder but the table of values."""
+    x = np.asarray(x, dtype=np.float64)
+    grid = e4m3_decode(np.arange(0x7F, dtype=np.uint8))            # 0 .. 448, increasing with the code
+    mag = np.minimum(np.abs(x), E4M3_MAX)
+    hi = np.clip(np.searchsorted(grid, mag, side='left'), 0, len(grid) - 1)
+    lo = np.maximum(hi - 1, 0)
+    d_lo, d_hi = mag - grid[lo], grid[hi] - mag
+    pick_hi = (d_hi < d_lo) | ((d_hi == d_lo) & (hi % 2 == 0))     # a tie goes to the code with an even mantissa
+    code = np.where(pick_hi, hi, lo).astype(np.uint8)
+    return np.where(np.signbit(x), code | 0x80, code).astype(np.uint8)
+
+
+def _round_bf16(x):
+    """float64 -> nearest bf16 value (ties to even), returned as float64."""
+    u = np.asarray(x, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000
+    return u.astype(np.uint32).view(np.float32).astype(np.float64)
+
+
+def quantize_latent_rows(rows, r):
+    """rows [..., r+dR] float64 -> (codes uint8 [..., r], k_pe float64 [..., dR] (bf16 values), scale float64 [...])."""
+    rows = np.asarray(rows, np.float64)
+    c, k = rows[..., :r], rows[..., r:]
+    amax = np.abs(c).max(axis=-1)
+    scale = np.where(amax > 0, amax / E4M3_MAX, 1.0).astype(np.float32).astype(np.float64)
+    codes = e4m3_encode(c / scale[..., None])
+    return codes, _round_bf16(k / scale[..., None]), scale
+
+
+def dequantize_latent_rows(codes, k_pe, scale):
+    """The rows the attention sees: [scale * decode(codes) ; scale * k_pe], float64."""
+    scale = np.asarray(scale, np.float64)[..., None]
+    return np.concatenate([scale * e4m3_decode(codes), scale * np.asarray(k_pe, np.float64)], axis=-1)
+
+
+def mla_decode_fp8_cache(q_nope, q_pe, w_uk, w_uv, codes, k_pe, scale, page_table, seqlens, softmax_scale, page_size=64,
+                         only=None):
+    """Eq. 9 over an FP8 latent cache: dequantise every row, then the MHA form above.
+
+    codes [num_pages, P, r] uint8, k_pe [num_pages, P, dR], scale [num_pages, P].  Rows that no sequence owns may hold
+    anything (NaN codes included): they are never gathered.
+    """
+    with np.errstate(invalid='ignore'):
+        cache = dequantize_latent_rows(codes, k_pe, scale)
+    return mla_decode_mha_form(q_nope, q_pe, w_uk, w_uv, cache, page_table, seqlens, softmax_scale, page_size, only)
+
+
+def latent_append_fp8(x, w_dkv_kr, positions, page_table, codes, k_pe, scale, r, theta=10000.0, page_size=64):
+    """Eq. 7 left, then the quantisation above, into the FP8 cache arrays (modified in place)."""
+    x = np.asarray(x, np.float64)
+    w = np.asarray(w_dkv_kr, np.float64)
+    for b in range(x.shape[0]):
+        y = w @ x[b]
+        y[r:] = rope(y[r:], int(positions[b]), theta)
+        page, off = append_slot(page_table[b], int(positions[b]), page_size)
+        codes[page, off], k_pe[page, off], scale[page, off] = quantize_latent_rows(y, r)
+    return codes, k_pe, scale
