@@ -36,6 +36,8 @@ def workloads():
     w['llama2-7b-mla_ragged_b32'] = (synth.LLAMA2_7B, synth.uniform_seqlens(32, 1024, 32768, 4), 4)
     w['llama2-7b-mla_b4_128k'] = (synth.LLAMA2_7B, [131072] * 4, 4)
     w['qwen2.5-72b-mla_b64_s2'] = (synth.QWEN25_72B, synth.uniform_seqlens(64, 2048, 8192, 5), 5)
+    for B in (16, 64, 128):      # the same shape over the FP8 latent cache (656 bytes a token instead of 1152)
+        w[f'llama2-7b-mla-fp8_b{B}_8k'] = (synth.LLAMA2_7B, [8192] * B, 6)
     return w
 
 
@@ -247,14 +249,22 @@ def measure(args, name, shape, seqlens, seed, rank, world, local, full):
     n_copies = args.cache_copies
     dc = synth.make_decode_case(shape, seqlens, replicas.rank_seed(seed, rank), device='cuda')
     ac = synth.make_append_case(shape, [L - S for L in seqlens], replicas.rank_seed(seed, rank) + 1, device='cuda')
-    caches = [dc['cache']] + [dc['cache'].clone() for _ in range(n_copies - 1)]
+    fp8 = '-fp8' in name
+    if fp8:   # the FP8 cache replaces the bf16 one: same page table, rows in the library's 656-byte format
+        first = synth.make_fp8_cache(shape, dc['cache'].shape[0], seed + 100, device='cuda')
+        dc['cache'] = None
+        caches = [first] + [first.clone() for _ in range(n_copies - 1)]
+        fp8_scratch = torch.empty(B * S * shape.row, dtype=torch.float32, device='cuda')
+        fp8_positions = torch.tensor([L - S for L in seqlens], dtype=torch.int32, device='cuda')
+    else:
+        caches = [dc['cache']] + [dc['cache'].clone() for _ in range(n_copies - 1)]
     # Weights rotate as well (their copies together exceed L2): in a whole model every other layer's weights pass
     # through L2 between two steps of this layer, so a step must find its own weights in HBM, not in L2.
     n_w = args.weight_copies
     weights = [(ac['w_dkv_kr'], dc['w_uk'], dc['w_uv'])] + [
         (ac['w_dkv_kr'].clone(), dc['w_uk'].clone(), dc['w_uv'].clone()) for _ in range(n_w - 1)]
     weight_bytes = sum(t.numel() * t.element_size() for t in weights[0])
-    params = binding.make_params(shape, B, dc['cache'].shape[0], dc['page_table'].shape[1], scale)
+    params = binding.make_params(shape, B, caches[0].shape[0], dc['page_table'].shape[1], scale)
     ws, lay = binding.alloc_workspace(params)
     out = torch.empty(B, S, H, shape.dv, dtype=torch.bfloat16, device='cuda')
     lse = torch.empty(B, S, H, dtype=torch.float32, device='cuda')
@@ -264,6 +274,14 @@ def measure(args, name, shape, seqlens, seed, rank, world, local, full):
     def step(i, ev=None):
         if ev is not None:
             binding.transmla_profile_decode_kernel(ev[0], ev[1])
+        if fp8:   # append, absorb + plan + split-KV decode, combine: five launches
+            w_dkv_kr, w_uk, w_uv = weights[i % n_w]
+            binding.transmla_latent_append_fp8(params, ac['x'], w_dkv_kr, fp8_positions, dc['page_table'], caches[i % n_copies],
+                                               fp8_scratch, status, stream)
+            binding.transmla_mla_decode_fp8(params, dc['q_nope'], dc['q_pe'], w_uk, caches[i % n_copies], dc['page_table'],
+                                            dc['seqlens'], ws, status, stream)
+            binding.transmla_mla_combine(params, ws, w_uv, out, lse, status, stream)
+            return
         binding.transmla_decode_step(params, ac['x'], dc['q_nope'], dc['q_pe'], dc['page_table'], dc['seqlens'],
                                      *weights[i % n_w], caches[i % n_copies], ws, out, lse,
                                      status, stream)
@@ -310,7 +328,7 @@ def measure(args, name, shape, seqlens, seed, rank, world, local, full):
     # Read-only streaming probe: the same pages through the same grid and TMA ring with nothing computed; its time is
     # the floor under the split-KV kernel for this workload (r = 512, dR = 64 only).
     probe_us = None
-    if shape.r == 512 and shape.dR == 64:
+    if shape.r == 512 and shape.dR == 64 and not fp8:
         probe = []
         for i in range(3 + 20):
             ev = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
@@ -348,7 +366,7 @@ def measure(args, name, shape, seqlens, seed, rank, world, local, full):
         d2h = h_out.numel() * 2 + h_lse.numel() * 4 + 4
         return e2e_s, h2d, d2h
 
-    e2e_s, h2d, d2h = end_to_end() if full else (float('nan'), 0, 0)   # skipped for the rows of the sweep
+    e2e_s, h2d, d2h = end_to_end() if full and not fp8 else (float('nan'), 0, 0)   # skipped for the rows of the sweep
 
     layer = None
     if args.layer and full:
@@ -387,7 +405,7 @@ def measure(args, name, shape, seqlens, seed, rank, world, local, full):
 
     tokens_per_step = B * S * world
     ms_step = ms_total / steps
-    cache_bytes = sum(seqlens) * shape.row * 2                       # live latent rows, read once
+    cache_bytes = sum(seqlens) * (synth.FP8_ROW_BYTES if fp8 else shape.row * 2)   # live latent rows, read once
     q_hat_bytes = B * S * H * shape.row * 2
     algo_bytes = cache_bytes + q_hat_bytes                           # per split-KV launch
     achieved = algo_bytes / (kernel_ms * 1e-3) / 1e9
@@ -403,7 +421,7 @@ def measure(args, name, shape, seqlens, seed, rank, world, local, full):
     line = {
         'metric': METRIC, 'value': replicas.whole_job_rate(B * S, steps, ms_total), 'unit': 'tokens/s', 'n_gpus': world,
         'steps': steps, 'warmup': max(args.warmup, 3), 'ms_per_step': ms_step, 'higher_is_better': True,
-        'scaling': 'weak', 'vs_baseline': None, 'dtype': 'bf16', 'data': 'synthetic',
+        'scaling': 'weak', 'vs_baseline': None, 'dtype': 'e4m3 cache, bf16/fp16 operands' if fp8 else 'bf16', 'data': 'synthetic',
         'config': {'workload': name, 'batch_per_gpu': B, 'q_len': S, 'heads': H, 'latent': shape.r, 'rope': shape.dR,
                    'cached_tokens_per_gpu': sum(seqlens), 'page_size': shape.page_size,
                    'num_partitions': lay.num_partitions, 'page_claims': claims,
@@ -425,7 +443,7 @@ def measure(args, name, shape, seqlens, seed, rank, world, local, full):
                                 'frac': tflops / tpeak, 'flops_per_launch': flops}},
         'e2e': {'value': replicas.whole_job_rate(B * S, steps, e2e_ms), 'unit': 'tokens/s',
                 'h2d_bytes_per_step': h2d, 'd2h_bytes_per_step': d2h, 'ms_per_step': e2e_ms / steps},
-        'gpu_launches': KERNELS_PER_STEP * steps,
+        'gpu_launches': (5 if fp8 else KERNELS_PER_STEP) * steps,
         'clocks': clocks,
     }
     if layer is not None:
@@ -446,7 +464,7 @@ def main():
     ap.add_argument('--layer', action='store_true', help='also time the whole layer step (queries, attention, W_O)')
     ap.add_argument('--q-lora-rank', type=int, default=0, help='low-rank queries for --layer (0: full rank)')
     ap.add_argument('--layer-weight-copies', type=int, default=6)
-    ap.add_argument('--sweep', default='llama2-7b-mla_b64_8k,llama2-7b-mla_b128_8k,qwen2.5-72b-mla_b64_s2',
+    ap.add_argument('--sweep', default='llama2-7b-mla_b64_8k,llama2-7b-mla_b128_8k,qwen2.5-72b-mla_b64_s2,llama2-7b-mla-fp8_b64_8k',
                     help='comma-separated workloads measured after the main one (1 GPU; empty: none)')
     args = ap.parse_args()
     w = workloads()

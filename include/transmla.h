@@ -57,6 +57,9 @@ typedef enum {
   TRANSMLA_ERR_ARCH = 7       /* the current device is not compute capability 10.x */
 } transmla_status_t;
 
+/* bytes of one token's row in the FP8 latent cache (r = 512, dR = 64): 512 e4m3 codes, 64 bf16, fp32 scale, padding */
+#define TRANSMLA_FP8_ROW_BYTES 656
+
 /* page-equivalents charged to a partition for every sequence it opens (split plan) */
 #define TRANSMLA_SEGMENT_COST_PAGES 2
 
@@ -290,6 +293,31 @@ transmla_status_t transmla_mla_attention_static(const transmla_params_t* params 
  * (device int32, required), a second wait returns immediately and the kernel ends; the context stays
  * usable.  cycles_out (device int64[2], may be NULL) receives the SM cycles spent in the two waits. */
 transmla_status_t transmla_selftest_bounded_wait(int32_t* dev_status, long long* cycles_out, void* stream);
+
+/* FP8 latent cache (the paper's abstract names FP8 quantisation as combinable with the method and gives no detail; the
+ * stored format is this library's own).  Only r = 512, dR = 64.  A token's row is TRANSMLA_FP8_ROW_BYTES = 656 bytes:
+ *     bytes   0..511   e4m3 codes (OCP 8-bit float: 1 sign, 4 exponent bits with bias 7, 3 mantissa bits, largest
+ *                      finite value 448, no infinities) of c_t / scale_t, nearest with ties to even
+ *     bytes 512..639   k^R_t / scale_t as 64 bf16 values
+ *     bytes 640..643   scale_t = max_i |c_t[i]| / 448 as fp32 (1.0 for an all-zero row); bytes 644..655 unused
+ * and the cache is [num_pages, P, 656] bytes, 128-byte aligned.  What the attention sees is the dequantised row
+ * scale_t * code, scale_t * (k^R_t / scale_t); results are Eq. 9 on those values.  |c| must stay below 65504 (the
+ * products run on fp16 copies of scale_t * code).
+ *
+ * transmla_latent_append_fp8: transmla_latent_append into such a cache.  `scratch` is device memory of at least
+ * B * S * (r + dR) * 4 bytes, 16-byte aligned (the rows in fp32 between the projection and the quantisation: a row's
+ * scale needs all of its values).  Two launches.
+ * transmla_mla_decode_fp8: transmla_mla_decode over such a cache; same workspace, and transmla_mla_combine finishes
+ * the step exactly as for a bf16 cache.  The scores run as native e4m3 products on the stored codes, with every
+ * absorbed query row split into two e4m3 terms (about the precision of its bf16 value). */
+transmla_status_t transmla_latent_append_fp8(const transmla_params_t* params /* host */, const void* x,
+                                             const void* w_dkv_kr, const int32_t* positions, const int32_t* page_table,
+                                             void* cache_fp8, void* scratch, size_t scratch_bytes, int32_t* dev_status,
+                                             void* stream);
+transmla_status_t transmla_mla_decode_fp8(const transmla_params_t* params /* host */, const void* q_nope, const void* q_pe,
+                                          const void* w_uk, const void* cache_fp8, const int32_t* page_table,
+                                          const int32_t* seqlens, void* workspace, size_t workspace_bytes,
+                                          int32_t* dev_status, void* stream);
 
 /* Whether transmla_mla_decode with these `params` hands pages to CTAs at run time (1) or keeps to the page ranges of
  * the split plan (0); see transmla_params_t.num_partitions.  With run-time claims the default path is not

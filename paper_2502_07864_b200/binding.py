@@ -15,7 +15,8 @@ EXPORTS = ('transmla_workspace_layout', 'transmla_latent_append', 'transmla_mla_
            'transmla_validate_tables', 'transmla_step_staging_bytes', 'transmla_decode_step_host',
            'transmla_decode_step', 'transmla_profile_decode_kernel', 'transmla_status_string',
            'transmla_static_workspace_capacity', 'transmla_mla_attention_static', 'transmla_selftest_bounded_wait',
-           'transmla_layer_scratch_bytes', 'transmla_layer_decode_step', 'transmla_stream_probe', 'transmla_page_claims_at_run_time')
+           'transmla_layer_scratch_bytes', 'transmla_layer_decode_step', 'transmla_stream_probe', 'transmla_page_claims_at_run_time', 'transmla_latent_append_fp8',
+           'transmla_mla_decode_fp8')
 
 
 class Params(ctypes.Structure):
@@ -74,6 +75,8 @@ def lib():
         L.transmla_selftest_bounded_wait.argtypes = [i32p, vp, vp]
         L.transmla_stream_probe.argtypes = [pp, vp, i32p, vp, sz, i32p, vp]
         L.transmla_page_claims_at_run_time.argtypes = [pp]
+        L.transmla_latent_append_fp8.argtypes = [pp, vp, vp, i32p, i32p, vp, vp, sz, i32p, vp]
+        L.transmla_mla_decode_fp8.argtypes = [pp, vp, vp, vp, vp, i32p, i32p, vp, sz, i32p, vp]
         L.transmla_layer_scratch_bytes.argtypes = [pp, ctypes.c_int32]
         L.transmla_layer_scratch_bytes.restype = sz
         L.transmla_layer_decode_step.argtypes = [pp, ctypes.POINTER(LayerWeights), vp, i32p, i32p, vp, vp, sz, vp, sz, vp,
@@ -207,6 +210,23 @@ def transmla_layer_decode_step(params, weights, x, page_table, seqlens, cache, w
 def transmla_selftest_bounded_wait(dev_status, cycles_out=None, stream=None):
     _check(lib().transmla_selftest_bounded_wait(_ptr(dev_status), _ptr(cycles_out), _stream(stream)),
            'transmla_selftest_bounded_wait')
+
+
+FP8_ROW_BYTES = 656
+
+
+def transmla_latent_append_fp8(params, x, w_dkv_kr, positions, page_table, cache_fp8, scratch, dev_status=None, stream=None):
+    _check(lib().transmla_latent_append_fp8(ctypes.byref(params), _ptr(x), _ptr(w_dkv_kr), _ptr(positions), _ptr(page_table),
+                                            _ptr(cache_fp8), _ptr(scratch), scratch.numel() * scratch.element_size(),
+                                            _ptr(dev_status), _stream(stream)), 'transmla_latent_append_fp8')
+
+
+def transmla_mla_decode_fp8(params, q_nope, q_pe, w_uk, cache_fp8, page_table, seqlens, workspace, dev_status=None,
+                            stream=None):
+    _check(lib().transmla_mla_decode_fp8(ctypes.byref(params), _ptr(q_nope), _ptr(q_pe), _ptr(w_uk), _ptr(cache_fp8),
+                                         _ptr(page_table), _ptr(seqlens), _ptr(workspace),
+                                         workspace.numel() * workspace.element_size(), _ptr(dev_status), _stream(stream)),
+           'transmla_mla_decode_fp8')
 
 
 def transmla_page_claims_at_run_time(params):

@@ -240,6 +240,55 @@ transmla_status_t transmla_mla_combine(const transmla_params_t* p, const void* w
   return e == cudaSuccess ? TRANSMLA_OK : TRANSMLA_ERR_CUDA;
 }
 
+transmla_status_t transmla_latent_append_fp8(const transmla_params_t* p, const void* x, const void* w_dkv_kr,
+                                             const int32_t* positions, const int32_t* page_table, void* cache_fp8,
+                                             void* scratch, size_t scratch_bytes, int32_t* dev_status, void* stream) {
+  transmla_status_t st = check_shape(p, true);
+  if (st != TRANSMLA_OK) return st;
+  if (!decode_fp8_supported(*p)) return TRANSMLA_ERR_SHAPE;
+  if (!x || !w_dkv_kr || !positions || !page_table || !cache_fp8 || !scratch) return TRANSMLA_ERR_NULL;
+  if (!aligned(x, 16) || !aligned(w_dkv_kr, 16) || !aligned(positions, 4) || !aligned(page_table, 4) ||
+      !aligned(cache_fp8, 128) || !aligned(scratch, 16) || !aligned(dev_status, 4))
+    return TRANSMLA_ERR_ALIGN;
+  const size_t need = static_cast<size_t>(p->batch) * p->q_len * (p->kv_lora_rank + p->qk_rope_dim) * sizeof(float);
+  if (scratch_bytes < need) return TRANSMLA_ERR_WORKSPACE;
+  st = check_device(nullptr);
+  if (st != TRANSMLA_OK) return st;
+  cudaError_t e = launch_append_fp8(*p, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w_dkv_kr),
+                                    positions, page_table, cache_fp8, static_cast<float*>(scratch), dev_status,
+                                    static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? TRANSMLA_OK : TRANSMLA_ERR_CUDA;
+}
+
+transmla_status_t transmla_mla_decode_fp8(const transmla_params_t* p, const void* q_nope, const void* q_pe,
+                                          const void* w_uk, const void* cache_fp8, const int32_t* page_table,
+                                          const int32_t* seqlens, void* workspace, size_t workspace_bytes,
+                                          int32_t* dev_status, void* stream) {
+  transmla_workspace_layout_t lay;
+  transmla_status_t st = check_decode_args(p, q_nope, q_pe, w_uk, cache_fp8, page_table, seqlens, workspace,
+                                           workspace_bytes, dev_status, &lay);
+  if (st != TRANSMLA_OK) return st;
+  if (!decode_fp8_supported(*p)) return TRANSMLA_ERR_SHAPE;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  char* ws = static_cast<char*>(workspace);
+  if (launch_absorb_plan(*p, lay.num_partitions, static_cast<const __nv_bfloat16*>(q_nope),
+                         static_cast<const __nv_bfloat16*>(q_pe), static_cast<const __nv_bfloat16*>(w_uk),
+                         reinterpret_cast<__nv_bfloat16*>(ws + lay.q_hat_offset), seqlens,
+                         reinterpret_cast<int32_t*>(ws + lay.cum_pages_offset),
+                         reinterpret_cast<int32_t*>(ws + lay.plan_offset), dev_status, s) != cudaSuccess)
+    return TRANSMLA_ERR_CUDA;
+  cudaEvent_t ev0 = tl_prof_start, ev1 = tl_prof_stop;
+  tl_prof_start = tl_prof_stop = nullptr;
+  if (ev0 != nullptr && cudaEventRecord(ev0, s) != cudaSuccess) return TRANSMLA_ERR_CUDA;
+  if (launch_decode_fp8(*p, lay.num_partitions, reinterpret_cast<__nv_bfloat16*>(ws + lay.q_hat_offset), cache_fp8, page_table,
+                        seqlens, reinterpret_cast<int32_t*>(ws + lay.cum_pages_offset),
+                        reinterpret_cast<int32_t*>(ws + lay.plan_offset), reinterpret_cast<float*>(ws + lay.partial_o_offset),
+                        reinterpret_cast<float*>(ws + lay.partial_lse_offset), dev_status, s) != cudaSuccess)
+    return TRANSMLA_ERR_CUDA;
+  if (ev1 != nullptr && cudaEventRecord(ev1, s) != cudaSuccess) return TRANSMLA_ERR_CUDA;
+  return TRANSMLA_OK;
+}
+
 int transmla_page_claims_at_run_time(const transmla_params_t* p) {
   transmla_workspace_layout_t lay;
   if (transmla_workspace_layout(p, &lay) != TRANSMLA_OK) return 0;

@@ -207,6 +207,13 @@ cudaError_t launch_decode_sm100(const transmla_params_t& p, int G, const __nv_bf
                                 const __nv_bfloat16* cache, const int32_t* page_table, const int32_t* seqlens,
                                 const int32_t* cum, const int32_t* plan, float* partial_o, float* partial_lse,
                                 int32_t* dev_status, cudaStream_t stream);
+bool decode_fp8_supported(const transmla_params_t& p);
+cudaError_t launch_decode_fp8(const transmla_params_t& p, int G, const __nv_bfloat16* q_hat, const void* cache_fp8,
+                              const int32_t* page_table, const int32_t* seqlens, const int32_t* cum, const int32_t* plan,
+                              float* partial_o, float* partial_lse, int32_t* dev_status, cudaStream_t stream);
+cudaError_t launch_append_fp8(const transmla_params_t& p, const __nv_bfloat16* x, const __nv_bfloat16* w, const int32_t* positions,
+                              const int32_t* page_table, void* cache_fp8, float* scratch, int32_t* dev_status,
+                              cudaStream_t stream);
 cudaError_t launch_stream_probe(const transmla_params_t& p, int G, const __nv_bfloat16* cache, const int32_t* page_table,
                                 const int32_t* cum, const int32_t* plan, int32_t* dev_status, cudaStream_t stream);
 cudaError_t launch_combine(const transmla_params_t& p, int G, const int32_t* cum, const float* partial_o,

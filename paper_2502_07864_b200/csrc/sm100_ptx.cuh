@@ -118,29 +118,31 @@ inline PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
   return fn;
 }
 
-// Tensor map of a dense row-major bf16 matrix [rows, cols] read in boxes of box_rows x 64 columns (128 bytes) with
-// the 128-byte swizzle.  Encoding one costs a driver call of about a microsecond and a decode step needs the same
+// Tensor map of a dense row-major matrix [rows, cols] (bf16, or bytes) read in boxes of box_rows x box_cols elements,
+// by default 64 bf16 columns (128 bytes) with the 128-byte swizzle.  Encoding one costs a driver call of about a microsecond and a decode step needs the same
 // two every time (the cache pool and the workspace do not move), so the last few are kept, keyed by device, base
 // address and geometry, behind a mutex.  A tensor map holds nothing but that address and geometry, so a cached one
 // stays right for as long as the key matches, whatever has happened to the memory in between.
+// kind: what the elements are and how a box is laid out in shared memory.
+enum { TMAP_BF16_SW128 = 0, TMAP_U8_SW128 = 1, TMAP_U8_PLAIN = 2 };
 struct TensorMapKey {
   int device;
   const void* base;
   uint64_t rows;
-  uint32_t cols, box_rows, box_cols;
+  uint32_t cols, box_rows, box_cols, kind;
   bool operator==(const TensorMapKey& o) const {
     return device == o.device && base == o.base && rows == o.rows && cols == o.cols && box_rows == o.box_rows &&
-           box_cols == o.box_cols;
+           box_cols == o.box_cols && kind == o.kind;
   }
 };
 inline bool tensor_map_2d(CUtensorMap* out, const void* base, uint64_t rows, uint32_t cols, uint32_t box_rows,
-                          uint32_t box_cols = 64) {
+                          uint32_t box_cols = 64, uint32_t kind = TMAP_BF16_SW128) {
   constexpr int kSlots = 16;
   struct Slot { TensorMapKey key; CUtensorMap map; uint64_t used; };
   static std::mutex mutex;
   static Slot slots[kSlots] = {};
   static uint64_t tick = 0;
-  TensorMapKey key = {current_device_slot(), base, rows, cols, box_rows, box_cols};
+  TensorMapKey key = {current_device_slot(), base, rows, cols, box_rows, box_cols, kind};
   std::lock_guard<std::mutex> lock(mutex);
   int victim = 0;
   for (int i = 0; i < kSlots; ++i) {
@@ -154,12 +156,13 @@ inline bool tensor_map_2d(CUtensorMap* out, const void* base, uint64_t rows, uin
   auto encode = encode_fn();
   if (encode == nullptr) return false;
   const cuuint64_t dims[2] = {cols, rows};
-  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(cols) * sizeof(__nv_bfloat16)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(cols) * (kind == TMAP_BF16_SW128 ? sizeof(__nv_bfloat16) : 1)};
   const cuuint32_t box[2] = {box_cols, box_rows};
   const cuuint32_t elem_strides[2] = {1, 1};
   CUtensorMap map;
-  if (encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, elem_strides,
-             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+  if (encode(&map, kind == TMAP_BF16_SW128 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 2,
+             const_cast<void*>(base), dims, strides, box, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE,
+             kind == TMAP_U8_PLAIN ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return false;
   slots[victim].key = key;

@@ -102,6 +102,28 @@ def make_decode_case(shape, seqlens, seed, pool_factor=1.2, device='cpu', nan_ta
     return case
 
 
+FP8_ROW_BYTES = 656   # 512 e4m3 codes, 64 bf16, one fp32 scale, 12 bytes unused
+
+
+def make_fp8_cache(shape, num_pages, seed, device='cpu'):
+    """A latent cache in the library's FP8 row format, [num_pages, P, 656] uint8, filled with seeded N(0,1) rows that
+    are rounded once to the storage format (as the bf16 cache is rounded once to bf16): per row scale = max|c| / 448,
+    codes = e4m3(c / scale) by torch's float8 cast, k_pe / scale in bf16.  r = 512, dR = 64."""
+    assert shape.r == 512 and shape.dR == 64
+    g = _gen(seed, device)
+    P = shape.page_size
+    out = torch.zeros((num_pages, P, FP8_ROW_BYTES), dtype=torch.uint8, device=device)
+    step = 2048
+    for i in range(0, num_pages, step):
+        n = min(step, num_pages - i)
+        rows = torch.randn((n, P, shape.row), generator=g, device=device, dtype=torch.float32)
+        scale = rows[..., :shape.r].abs().amax(dim=-1, keepdim=True) / 448.0
+        out[i:i + n, :, :shape.r] = (rows[..., :shape.r] / scale).to(torch.float8_e4m3fn).view(torch.uint8)
+        out[i:i + n, :, shape.r:shape.r + 2 * shape.dR] = (rows[..., shape.r:] / scale).to(torch.bfloat16).view(torch.uint8).view(n, P, -1)
+        out[i:i + n, :, 640:644] = scale.contiguous().view(torch.uint8).view(n, P, 4)
+    return out
+
+
 def make_append_case(shape, positions, seed, device='cpu'):
     """Inputs of one append step: x [B, S, D] ~ N(0,1), w_dkv_kr [r+dR, D] ~ N(0, 1/sqrt(D)), bf16;
     positions [B] = position of each sequence's first new token."""

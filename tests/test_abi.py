@@ -15,7 +15,7 @@ def test_library_exports_every_declared_symbol():
     build.build()
     L = binding.lib()
     header = open(os.path.join(ROOT, 'include', 'transmla.h')).read()
-    declared = set(re.findall(r'\b(transmla_[a-z_]+)\s*\(', header))
+    declared = set(re.findall(r'\b(transmla_[a-z0-9_]+)\s*\(', header))
     assert declared, 'no declarations found'
     for name in declared:
         assert hasattr(L, name), f'{name} declared in transmla.h but not exported'
