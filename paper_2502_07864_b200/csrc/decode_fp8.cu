@@ -7,8 +7,8 @@
 //     queries are split, row by row, into two e4m3 terms q ~ sq * (hi + lo) when they are moved into tensor memory
 //     (two terms carry about the 8 bits a bf16 query has); the rope part runs as bf16 products on k^R / scale and
 //     q^R / sq.  All of it lands in one accumulator and a score is sq * scale_j times that sum.
-//   - products: four more warps turn the codes of a page into scale_j * code as fp16 (exact product of an fp16
-//     scale... rounded once, 2^-11) in a second buffer with the layout the bf16 kernel reads its pages in, and
+//   - products: four more warps turn the codes of a page into scale_j * code as fp16 (the code's fp16 image is exact,
+//     the product with the fp16-rounded scale is rounded once more) in a second buffer with the layout the bf16 kernel reads its pages in, and
 //     zero-fill the rows beyond the sequence; P is fp16 too (operands of one product must agree in type).
 //   - a page's stage goes back to the TMA warp when three parties are done with it: the scores, the converters,
 //     and the softmax warps (they read the scales).
@@ -350,10 +350,10 @@ decode_fp8_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_co
     } else if (warp >= 7) {
       // ======================================================================== converters (warps 7-10)
       // Per page: scale_j * code -> fp16 into the V buffer, in the layout of a bf16 page's latent sub-tiles (64
-      // tokens x 64 columns, 128-byte rows, 128-byte swizzle); rows beyond the sequence become zeros.  Thread c
-      // takes half of row c / 2.  They hand a query item back too (their third of it), so that no stage can be
+      // tokens x 64 columns, 128-byte rows, 128-byte swizzle); rows beyond the sequence become zeros.  They hand a
+      // query item back too (their third of it), so that no stage can be
       // used twice before they have seen it.
-      const int c = tid - 224, r = c >> 1, half = c & 1;
+      const int c = tid - 224;
       int g = 0, n = 0, L_seg = 0;
       while (true) {
         const int stage = g % kStages, use = g / kStages;
@@ -373,14 +373,15 @@ decode_fp8_kernel(const __grid_constant__ CUtensorMap cache_map, const __grid_co
         const unsigned char* st = sm + kOffStage + stage * kStageBytes;
         unsigned char* vb = sm + kOffV;
         const int valid = m.z != 0 ? min(kPage, L_seg - m.y * kPage) : 0;  // rows [valid, 64) must read as zero
-        const __half sc = __float2half_rn(r < valid ? *reinterpret_cast<const float*>(st + kOffScale + r * 16) : 0.f);
-        const __half2 sc2 = __half2half2(sc);
+        // 16 rounds; in a round a warp takes 4 consecutive rows x the 8 16-byte chunks of one 128-code sub-tile, so that
+        // its loads sweep whole 128-byte rows (the swizzle only permutes the chunks inside a row)
+#pragma unroll 1
+        for (int rblk = 0; rblk < 4; ++rblk) {
+          const int r = rblk * 16 + (c >> 3), j = c & 7;
+          const __half2 sc2 = __half2half2(__float2half_rn(r < valid ? *reinterpret_cast<const float*>(st + kOffScale + r * 16) : 0.f));
 #pragma unroll
-        for (int tile = 0; tile < 2; ++tile) {
-          const int ct = half * 2 + tile;  // code sub-tile: columns 128 ct .. 128 ct + 127
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {    // 16 codes at a time
-            uint4 x = *reinterpret_cast<const uint4*>(st + ct * kSubTileBytes + r * 128 + ((j ^ (r & 7)) << 4));
+          for (int ct = 0; ct < kCodeTiles; ++ct) {  // code sub-tile: columns 128 ct .. 128 ct + 127
+            const uint4 x = *reinterpret_cast<const uint4*>(st + ct * kSubTileBytes + r * 128 + ((j ^ (r & 7)) << 4));
             const uint32_t w[4] = {x.x, x.y, x.z, x.w};
             uint32_t o[8];
 #pragma unroll
