@@ -175,11 +175,11 @@ def run_reference(args, name, shape, seqlens, seed):
     }))
 
 
-def kernel_source_hash():
+def kernel_source_hash(fp8=False):
     """Hash of the sources the split-KV kernel is compiled from; ties an ncu capture to the code it was taken on."""
     import hashlib
     h = hashlib.sha256()
-    for f in ('decode_sm100.cu', 'common.cuh', 'sm100_ptx.cuh'):
+    for f in ('decode_fp8.cu' if fp8 else 'decode_sm100.cu', 'common.cuh', 'sm100_ptx.cuh'):
         h.update(open(os.path.join(ROOT, 'paper_2502_07864_b200', 'csrc', f), 'rb').read())
     return h.hexdigest()[:16]
 
@@ -187,7 +187,9 @@ def kernel_source_hash():
 def traffic_from_profile(name):
     """dram__bytes_read.sum + dram__bytes_write.sum of one split-KV launch, from the ncu summary under profiles/ for
     this workload; None when there is none or when the kernel's sources have changed since the capture."""
-    path = os.path.join(ROOT, 'profiles', f'decode_sm100_{name.replace("-mla", "")}.md')
+    fp8 = '-fp8' in name
+    kernel = 'decode_fp8' if fp8 else 'decode_sm100'
+    path = os.path.join(ROOT, 'profiles', f'{kernel}_{name.replace("-mla", "").replace("-fp8", "")}.md')
     try:
         text = open(path).read()
     except OSError:
@@ -197,7 +199,7 @@ def traffic_from_profile(name):
         if line.startswith('traffic_bytes_per_launch:') or line.startswith('kernel_source_hash:'):
             k, v = line.split(':', 1)
             vals[k] = v.strip()
-    if vals.get('kernel_source_hash') != kernel_source_hash() or 'traffic_bytes_per_launch' not in vals:
+    if vals.get('kernel_source_hash') != kernel_source_hash(fp8) or 'traffic_bytes_per_launch' not in vals:
         return None
     return float(vals['traffic_bytes_per_launch'])
 
