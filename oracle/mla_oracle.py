@@ -20,6 +20,10 @@ itself pinned to torch's scaled_dot_product_attention (Sec. 4.1, App. A.2.1), or
 re-basing of the latent (App. D.2), key/value balancing (Eq. 19), page-permutation invariance,
 partition invariance of split + combine, brute-force restatement of the split plan.
 
+Prefill (decompress_kv): ordinary multi-head attention (the routine pinned to torch) over its output
+equals mla_decode_mha_form, and a chunk of S query positions equals S single-position calls over the
+growing prefix.
+
 FP8 latent cache (end of the file): the e4m3 format is pinned to the values of its published
 definition and to torch's float8_e4m3fn conversions, the quantiser to its error bound and to exact
 round trips of representable rows, the attention over an FP8 cache to Eq. 9 over the dequantised rows
@@ -147,6 +151,24 @@ def mla_decode_mha_form(q_nope, q_pe, w_uk, w_uv, cache, page_table, seqlens, sc
         out[b, s, h] = (e / e.sum()) @ v
         lse[b, s, h] = m + np.log(e.sum())
     return out, lse
+
+
+# --------------------------------------------------------------------------------------------
+# Prefill in the MHA form (Sec. 3.3, Eq. 8 and Eq. 9 left): a chunk of S query positions per sequence is
+# what mla_decode_mha_form computes for that S; the library materialises the decompressed keys and
+# values first, which is this function.
+# --------------------------------------------------------------------------------------------
+def decompress_kv(cache, page_row, n, w_uk, w_uv, page_size=64):
+    """k^C_{j,h} = W_UK_h c_j and v_{j,h} = W_UV_h c_j (Eq. 8) for tokens 0..n-1 of one sequence.
+
+    Returns k_c [n, H, dn], v [n, H, dv] and the stored rotated keys k^R [n, dR] (shared by the heads).
+    """
+    r = w_uk.shape[2]
+    rows = gather_latent(cache, page_row, n, page_size)
+    c, k_r = rows[:, :r], rows[:, r:]
+    k_c = np.stack([c @ np.asarray(w_uk[h], np.float64).T for h in range(w_uk.shape[0])], axis=1)
+    v = np.stack([c @ np.asarray(w_uv[h], np.float64).T for h in range(w_uv.shape[0])], axis=1)
+    return k_c, v, k_r
 
 
 # --------------------------------------------------------------------------------------------

@@ -443,6 +443,42 @@ def test_layer_step_with_two_new_tokens_equals_two_single_token_steps():
     assert np.abs(swapped[:, ::-1] - y2).max() > 1e-3
 
 
+def test_decompressed_keys_and_values_under_ordinary_attention_give_the_mha_form():
+    # Eq. 8 + Eq. 9 left: per head the key is [W_UK_h c ; k^R] and the value W_UV_h c; ordinary multi-head
+    # attention (grouped_attention with g = h, itself pinned to torch) over them is the definition
+    rng = np.random.default_rng(41)
+    H, dn, dR, dv, r, P = 4, 8, 4, 6, 10, 4
+    L = 11
+    cache = rng.standard_normal((5, P, r + dR))
+    table = np.array([[3, 0, 4, 1]])
+    w_uk, w_uv = rng.standard_normal((H, dn, r)), rng.standard_normal((H, dv, r))
+    q_nope, q_pe = rng.standard_normal((1, 1, H, dn)), rng.standard_normal((1, 1, H, dR))
+    k_c, v, k_r = orc.decompress_kv(cache, table[0], L, w_uk, w_uv, P)
+    assert k_c.shape == (L, H, dn) and v.shape == (L, H, dv) and k_r.shape == (L, dR)
+    # token 6 lives in page table[0][1] = 0, row 2
+    assert np.allclose(k_c[6, 2], w_uk[2] @ cache[0, 2, :r], atol=TOL) and np.array_equal(k_r[6], cache[0, 2, r:])
+    k = np.concatenate([k_c, np.repeat(k_r[:, None, :], H, axis=1)], axis=2)
+    got = orc.grouped_attention(np.concatenate([q_nope[0, 0], q_pe[0, 0]], axis=1), k, v, 0.3)
+    want, _ = orc.mla_decode_mha_form(q_nope, q_pe, w_uk, w_uv, cache, table, [L], 0.3, page_size=P)
+    assert np.allclose(got, want[0, 0], atol=TOL)
+
+
+def test_a_chunk_of_query_positions_equals_single_positions_over_the_growing_prefix():
+    # chunked prefill: position s of S sees the prefix that a one-token step at length L - S + 1 + s sees
+    rng = np.random.default_rng(42)
+    H, dn, dR, dv, r, P = 3, 8, 4, 6, 10, 4
+    S, L = 7, 13
+    cache = rng.standard_normal((6, P, r + dR))
+    table = np.array([[5, 2, 0, 3]])
+    w_uk, w_uv = rng.standard_normal((H, dn, r)), rng.standard_normal((H, dv, r))
+    q_nope, q_pe = rng.standard_normal((1, S, H, dn)), rng.standard_normal((1, S, H, dR))
+    out, lse = orc.mla_decode_mha_form(q_nope, q_pe, w_uk, w_uv, cache, table, [L], 0.4, page_size=P)
+    for s in range(S):
+        o1, l1 = orc.mla_decode_mha_form(q_nope[:, s:s + 1], q_pe[:, s:s + 1], w_uk, w_uv, cache, table,
+                                         [L - S + 1 + s], 0.4, page_size=P)
+        assert np.allclose(out[0, s], o1[0, 0], atol=TOL) and np.allclose(lse[0, s], l1[0, 0], atol=TOL)
+
+
 def test_low_rank_queries_and_folded_output_projection():
     # Eq. 8 right: low-rank queries equal full-rank ones with W = W_U{Q,R} W_DQ; App. A.2.2: folding the block
     # diagonal of W_UV into W_O gives the same y from the latent-space outputs.
