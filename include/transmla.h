@@ -319,6 +319,37 @@ transmla_status_t transmla_mla_decode_fp8(const transmla_params_t* params /* hos
                                           const int32_t* seqlens, void* workspace, size_t workspace_bytes,
                                           int32_t* dev_status, void* stream);
 
+/* Prefill in the MHA form (Sec. 3.3: the compute-bound paradigm; Eq. 8 and Eq. 9 left).  For a chunk of S = q_len
+ * query positions per sequence - the last S of the L_b cached tokens, position s sees tokens [0, L_b - S + s] - the
+ * keys and values are decompressed once, k^C_{j,h} = W_UK_h c_j and v_{j,h} = W_UV_h c_j (Eq. 8), and ordinary causal
+ * attention runs per head on  z = q_nope . k^C + q_pe . k^R  (Eq. 9 left).  Same result as transmla_mla_decode +
+ * transmla_mla_combine for the same arguments; it costs 2 * r * (dn + dv) FLOPs per token and head once, instead of
+ * the absorbed form's wider products for every query row, and pays from a few hundred query positions per sequence
+ * on.  Only r = 512, dR = 64, dn = dv = 128 (TRANSMLA_ERR_SHAPE otherwise); q_len up to 2^20 (the limit
+ * S*H <= 1024 of the decode calls does not apply); num_partitions is ignored.
+ *   scratch: device, 128-byte aligned, at least transmla_prefill_scratch_bytes(params) bytes =
+ *     num_pages * P * H * (dn + dv) * 2: the decompressed store, row page*P + slot = [H][k^C (dn) | v (dv)] bf16,
+ *     written for every page that the page table names for tokens < L_b (rows of tokens >= L_b as zeros).
+ *   transmla_prefill_decompress fills it (one launch), transmla_prefill_attention reads it (one launch; `cache` is
+ *     read again for k^R), transmla_mla_prefill does both.  A store filled once serves any number of chunks over
+ *     the same cached tokens.
+ *   q_nope [B,S,H,dn], q_pe [B,S,H,dR] (rotated), w_uk [H,dn,r], w_uv [H,dv,r], cache, page_table, seqlens,
+ *   out [B,S,H,dv] bf16, lse [B,S,H] fp32 (may be NULL), dev_status: device, as in transmla_mla_decode.
+ * Errors as for the decode calls; bad page indices and lengths are reported through *dev_status. */
+size_t transmla_prefill_scratch_bytes(const transmla_params_t* params /* host */);
+transmla_status_t transmla_prefill_decompress(const transmla_params_t* params /* host */, const void* cache,
+                                              const int32_t* page_table, const int32_t* seqlens, const void* w_uk,
+                                              const void* w_uv, void* scratch, size_t scratch_bytes, int32_t* dev_status,
+                                              void* stream);
+transmla_status_t transmla_prefill_attention(const transmla_params_t* params /* host */, const void* q_nope, const void* q_pe,
+                                             const void* cache, const void* scratch, size_t scratch_bytes,
+                                             const int32_t* page_table, const int32_t* seqlens, void* out, float* lse,
+                                             int32_t* dev_status, void* stream);
+transmla_status_t transmla_mla_prefill(const transmla_params_t* params /* host */, const void* q_nope, const void* q_pe,
+                                       const void* w_uk, const void* w_uv, const void* cache, const int32_t* page_table,
+                                       const int32_t* seqlens, void* scratch, size_t scratch_bytes, void* out, float* lse,
+                                       int32_t* dev_status, void* stream);
+
 /* Whether transmla_mla_decode with these `params` hands pages to CTAs at run time (1) or keeps to the page ranges of
  * the split plan (0); see transmla_params_t.num_partitions.  With run-time claims the default path is not
  * bit-stable from run to run (results agree to fp32 rounding); pass the partition count that

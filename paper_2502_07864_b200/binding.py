@@ -16,7 +16,8 @@ EXPORTS = ('transmla_workspace_layout', 'transmla_latent_append', 'transmla_mla_
            'transmla_decode_step', 'transmla_profile_decode_kernel', 'transmla_status_string',
            'transmla_static_workspace_capacity', 'transmla_mla_attention_static', 'transmla_selftest_bounded_wait',
            'transmla_layer_scratch_bytes', 'transmla_layer_decode_step', 'transmla_stream_probe', 'transmla_page_claims_at_run_time', 'transmla_latent_append_fp8',
-           'transmla_mla_decode_fp8')
+           'transmla_mla_decode_fp8', 'transmla_prefill_scratch_bytes', 'transmla_prefill_decompress',
+           'transmla_prefill_attention', 'transmla_mla_prefill')
 
 
 class Params(ctypes.Structure):
@@ -77,6 +78,11 @@ def lib():
         L.transmla_page_claims_at_run_time.argtypes = [pp]
         L.transmla_latent_append_fp8.argtypes = [pp, vp, vp, i32p, i32p, vp, vp, sz, i32p, vp]
         L.transmla_mla_decode_fp8.argtypes = [pp, vp, vp, vp, vp, i32p, i32p, vp, sz, i32p, vp]
+        L.transmla_prefill_scratch_bytes.argtypes = [pp]
+        L.transmla_prefill_scratch_bytes.restype = sz
+        L.transmla_prefill_decompress.argtypes = [pp, vp, i32p, i32p, vp, vp, vp, sz, i32p, vp]
+        L.transmla_prefill_attention.argtypes = [pp, vp, vp, vp, vp, sz, i32p, i32p, vp, vp, i32p, vp]
+        L.transmla_mla_prefill.argtypes = [pp, vp, vp, vp, vp, vp, i32p, i32p, vp, sz, vp, vp, i32p, vp]
         L.transmla_layer_scratch_bytes.argtypes = [pp, ctypes.c_int32]
         L.transmla_layer_scratch_bytes.restype = sz
         L.transmla_layer_decode_step.argtypes = [pp, ctypes.POINTER(LayerWeights), vp, i32p, i32p, vp, vp, sz, vp, sz, vp,
@@ -227,6 +233,36 @@ def transmla_mla_decode_fp8(params, q_nope, q_pe, w_uk, cache_fp8, page_table, s
                                          _ptr(page_table), _ptr(seqlens), _ptr(workspace),
                                          workspace.numel() * workspace.element_size(), _ptr(dev_status), _stream(stream)),
            'transmla_mla_decode_fp8')
+
+
+def transmla_prefill_scratch_bytes(params):
+    return int(lib().transmla_prefill_scratch_bytes(ctypes.byref(params)))
+
+
+def _nbytes(t):
+    return t.numel() * t.element_size()
+
+
+def transmla_prefill_decompress(params, cache, page_table, seqlens, w_uk, w_uv, scratch, dev_status=None, stream=None):
+    _check(lib().transmla_prefill_decompress(ctypes.byref(params), _ptr(cache), _ptr(page_table), _ptr(seqlens), _ptr(w_uk),
+                                             _ptr(w_uv), _ptr(scratch), _nbytes(scratch), _ptr(dev_status), _stream(stream)),
+           'transmla_prefill_decompress')
+
+
+def transmla_prefill_attention(params, q_nope, q_pe, cache, scratch, page_table, seqlens, out, lse=None, dev_status=None,
+                               stream=None):
+    _check(lib().transmla_prefill_attention(ctypes.byref(params), _ptr(q_nope), _ptr(q_pe), _ptr(cache), _ptr(scratch),
+                                            _nbytes(scratch), _ptr(page_table), _ptr(seqlens), _ptr(out), _ptr(lse),
+                                            _ptr(dev_status), _stream(stream)),
+           'transmla_prefill_attention')
+
+
+def transmla_mla_prefill(params, q_nope, q_pe, w_uk, w_uv, cache, page_table, seqlens, scratch, out, lse=None,
+                         dev_status=None, stream=None):
+    _check(lib().transmla_mla_prefill(ctypes.byref(params), _ptr(q_nope), _ptr(q_pe), _ptr(w_uk), _ptr(w_uv), _ptr(cache),
+                                      _ptr(page_table), _ptr(seqlens), _ptr(scratch), _nbytes(scratch), _ptr(out), _ptr(lse),
+                                      _ptr(dev_status), _stream(stream)),
+           'transmla_mla_prefill')
 
 
 def transmla_page_claims_at_run_time(params):
