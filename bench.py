@@ -38,6 +38,8 @@ def workloads():
     w['qwen2.5-72b-mla_b64_s2'] = (synth.QWEN25_72B, synth.uniform_seqlens(64, 2048, 8192, 5), 5)
     for B in (16, 64, 128):      # the same shape over the FP8 latent cache (656 bytes a token instead of 1152)
         w[f'llama2-7b-mla-fp8_b{B}_8k'] = (synth.LLAMA2_7B, [8192] * B, 6)
+    for S in (128, 512, 2048, 8192):   # prefill in the MHA form: a chunk of S query positions over 8192 cached tokens
+        w[f'llama2-7b-mla_prefill_b4_8k_s{S}'] = (synth.MLAShape(H=32, dn=128, dR=64, dv=128, r=512, D=4096, S=S), [8192] * 4, 8)
     return w
 
 
@@ -230,8 +232,10 @@ def run_ours(args, name, shape, seqlens, seed):
                 if other and other != name:
                     sh, sl, sd = workloads()[other]
                     row = measure(args, other, sh, sl, sd, rank, world, local, full=False)
-                    line['sweep'].append({k: row[k] for k in ('config', 'ms_per_step', 'value', 'decode_kernel_us',
-                                                               'cache_gbs_pct_of_8tbs', 'roofline', 'clocks')})
+                    keep = ('config', 'ms_per_step', 'value', 'decode_kernel_us', 'cache_gbs_pct_of_8tbs', 'roofline', 'clocks')
+                    if 'prefill' in row:   # a prefill row carries its own metric and the two kernels' figures
+                        keep += ('metric', 'unit', 'prefill')
+                    line['sweep'].append({k: row[k] for k in keep})
         if world == 1 and not args.no_cpu_baseline:
             line['cpu_baseline'] = cpu_baseline(shape, seqlens, seed, (shape.dn + shape.dR) ** -0.5)
         print(json.dumps(line))
@@ -239,7 +243,88 @@ def run_ours(args, name, shape, seqlens, seed):
         dist.destroy_process_group()
 
 
+def measure_prefill(args, name, shape, seqlens, seed, rank, world, local):
+    """A prefill workload: one step = decompress the cached tokens (Eq. 8) + causal attention of the chunk (Eq. 9
+    left), two launches.  Both are dense contractions: the roofline is the measured bf16 GEMM rate."""
+    import torch
+    from paper_2502_07864_b200 import binding, replicas, synth
+    B, S, H = len(seqlens), shape.S, shape.H
+    stream = torch.cuda.current_stream()
+    n_copies = 2
+    case = synth.make_decode_case(shape, seqlens, seed, device='cuda')
+    caches = [case['cache']] + [case['cache'].clone() for _ in range(n_copies - 1)]
+    params = binding.make_params(shape, B, case['cache'].shape[0], case['page_table'].shape[1], (shape.dn + shape.dR) ** -0.5)
+    scratch = torch.empty(binding.transmla_prefill_scratch_bytes(params) // 2, dtype=torch.bfloat16, device='cuda')
+    status = torch.zeros(1, dtype=torch.int32, device='cuda')
+    out = torch.empty(B, S, H, shape.dv, dtype=torch.bfloat16, device='cuda')
+    lse = torch.empty(B, S, H, dtype=torch.float32, device='cuda')
+    steps = max(3, min(args.steps, 20))
+
+    def step(i):
+        binding.transmla_mla_prefill(params, case['q_nope'], case['q_pe'], case['w_uk'], case['w_uv'], caches[i % n_copies],
+                                     case['page_table'], case['seqlens'], scratch, out, lse, status, stream)
+
+    for i in range(3):
+        step(i)
+    replicas.barrier('cuda')
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local) if rank == 0 else None
+    t0 = time.perf_counter()
+    e0.record(stream)
+    for i in range(steps):
+        step(i)
+    e1.record(stream)
+    replicas.barrier('cuda')
+    t1 = time.perf_counter()
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop(t0, t1) if sampler else None
+    parts = {'decompress': [], 'attention': []}
+    for i in range(5):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        ev[0].record(stream)
+        binding.transmla_prefill_decompress(params, caches[i % n_copies], case['page_table'], case['seqlens'], case['w_uk'],
+                                            case['w_uv'], scratch, status, stream)
+        ev[1].record(stream)
+        binding.transmla_prefill_attention(params, case['q_nope'], case['q_pe'], caches[i % n_copies], scratch,
+                                           case['page_table'], case['seqlens'], out, lse, status, stream)
+        ev[2].record(stream)
+        torch.cuda.synchronize()
+        parts['decompress'].append(ev[0].elapsed_time(ev[1]))
+        parts['attention'].append(ev[1].elapsed_time(ev[2]))
+    assert int(status.item()) == 0
+    (ms_total,) = replicas.max_over_ranks([ms_total], device='cuda')
+    if rank != 0:
+        return None
+    dec_ms, att_ms = statistics.median(parts['decompress']), statistics.median(parts['attention'])
+    f_dec = 2.0 * shape.r * H * (shape.dn + shape.dv) * sum(seqlens)
+    vis = sum(max(0, L - (S - 1 - s)) for L in seqlens for s in range(S))        # visible (query, token) pairs per head
+    f_att = 2.0 * (shape.dn + shape.dR + shape.dv) * H * vis
+    tpeak, tpeak_kind = measured_tensor_peak()
+    top, top_ms, top_f = ('prefill attention', att_ms, f_att) if att_ms >= dec_ms else ('prefill decompress', dec_ms, f_dec)
+    ms_step = ms_total / steps
+    return {
+        'metric': 'MHA-form prefill tokens/s (chunk of S query positions per sequence over the paged latent cache)',
+        'value': replicas.whole_job_rate(B * S, steps, ms_total), 'unit': 'tokens/s', 'n_gpus': world, 'steps': steps, 'warmup': 3,
+        'ms_per_step': ms_step, 'higher_is_better': True, 'scaling': 'weak', 'vs_baseline': None, 'dtype': 'bf16',
+        'data': 'synthetic',
+        'config': {'workload': name, 'batch_per_gpu': B, 'q_len': S, 'heads': H, 'latent': shape.r, 'rope': shape.dR,
+                   'cached_tokens_per_gpu': sum(seqlens), 'page_size': shape.page_size,
+                   'l2': f'inputs larger than L2: decompressed store {scratch.numel() * 2 / 1e6:.0f} MB, cache rotates over '
+                         f'{n_copies} copies', 'parallelism': f'replicas x{world}, no data-path collective'},
+        'decode_kernel_us': None, 'cache_gbs_pct_of_8tbs': None,
+        'prefill': {'decompress_us': dec_ms * 1e3, 'decompress_tflops': f_dec / dec_ms / 1e9,
+                    'attention_us': att_ms * 1e3, 'attention_tflops': f_att / att_ms / 1e9,
+                    'flops_decompress': f_dec, 'flops_attention': f_att},
+        'roofline': {'bound': 'tensor', 'kernel': top, 'achieved': top_f / top_ms / 1e9, 'peak': tpeak, 'unit': 'TFLOP/s',
+                     'frac': top_f / top_ms / 1e9 / tpeak, 'peak_kind': f'{tpeak_kind} bf16 GEMM', 'traffic': None,
+                     'flops_per_launch': top_f},
+        'gpu_launches': 2 * steps, 'clocks': clocks,
+    }
+
+
 def measure(args, name, shape, seqlens, seed, rank, world, local, full):
+    if '_prefill_' in name:
+        return measure_prefill(args, name, shape, seqlens, seed, rank, world, local)
     """One workload: whole-step time over args.steps steps, split-KV kernel time, read-probe ceiling, and (full) the
     host-buffer end-to-end figure and the optional layer step.  Returns the JSON line as a dict (rank 0)."""
     import torch
@@ -466,7 +551,8 @@ def main():
     ap.add_argument('--layer', action='store_true', help='also time the whole layer step (queries, attention, W_O)')
     ap.add_argument('--q-lora-rank', type=int, default=0, help='low-rank queries for --layer (0: full rank)')
     ap.add_argument('--layer-weight-copies', type=int, default=6)
-    ap.add_argument('--sweep', default='llama2-7b-mla_b64_8k,llama2-7b-mla_b128_8k,qwen2.5-72b-mla_b64_s2,llama2-7b-mla-fp8_b64_8k',
+    ap.add_argument('--sweep', default='llama2-7b-mla_b64_8k,llama2-7b-mla_b128_8k,qwen2.5-72b-mla_b64_s2,llama2-7b-mla-fp8_b64_8k,'
+                            'llama2-7b-mla_prefill_b4_8k_s2048',
                     help='comma-separated workloads measured after the main one (1 GPU; empty: none)')
     args = ap.parse_args()
     w = workloads()
