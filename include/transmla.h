@@ -68,6 +68,7 @@ typedef enum {
 #define TRANSMLA_DEV_BAD_PAGE 1
 #define TRANSMLA_DEV_TIMEOUT 2
 #define TRANSMLA_DEV_BAD_LEN 4
+#define TRANSMLA_DEV_NUMERIC 8 /* conversion calls: an eigen-iteration did not converge, or a Gram matrix was singular */
 
 typedef struct {
   int32_t hidden_dim;        /* D; used by the append only */
@@ -349,6 +350,51 @@ transmla_status_t transmla_mla_prefill(const transmla_params_t* params /* host *
                                        const void* w_uk, const void* w_uv, const void* cache, const int32_t* page_table,
                                        const int32_t* seqlens, void* scratch, size_t scratch_bytes, void* out, float* lse,
                                        int32_t* dev_status, void* stream);
+
+/* Conversion of a GQA layer to MLA on calibration activations (Sec. 4.2, 4.3; App. B, C, D).  A one-off per model,
+ * not part of the decode step.  Every matrix here is fp32, dense, row-major, device memory, 16-byte aligned; the
+ * calls enqueue on `stream`, allocate nothing and report numerical trouble through TRANSMLA_DEV_NUMERIC in
+ * *dev_status.  Index conventions: the merged key of Sec. 4.1 has g*d entries, entry (j, c) = j*d + c for original
+ * head j and dimension c; RoPE pair l of a head is (2l, 2l+1) = (real, imaginary).  `fold` = M of App. C: group G
+ * holds frequencies G*M .. G*M+M-1 and has g*M real and g*M imaginary entries, entry i = p*g + j for frequency
+ * G*M + p and head j.
+ *   transmla_conv_gemm: C[M,N] = alpha * op(A) op(B); op(A) = A [M,K] (ta = 0) or the transpose of A [K,M]
+ *     (ta = 1), op(B) from B [K,N] (tb = 0) or B [N,K] (tb = 1); lda/ldb/ldc are row strides in elements.  Serves
+ *     the calibration activations (K = X W^T), second moments (Z^T Z) and the low-rank rewrite of App. D.2
+ *     (W_DKV' = R^T W_DKV, W_UKV' = W_UKV R).
+ *   transmla_conv_rorope_covariance: App. B's sigma_x + sigma_y per frequency group from key activations
+ *     K [n, g*d]: cov [d/2/fold, g*fold, g*fold].  scratch: transmla_conv_rorope_scratch_bytes(n, g, d, fold).
+ *     g*fold <= 128.
+ *   transmla_conv_sym_eig: eigenvalues (descending) and eigenvectors (columns of eigvecs [batch, m, m]) of `batch`
+ *     symmetric matrices a [batch, m, m], m <= 128 (cyclic Jacobi).  App. B: U_l is eigvecs of cov[l].
+ *   transmla_conv_rorope_apply: Eq. 18's rotation of the rows of X [g*d, C] (W^K, or merged queries/keys as
+ *     columns) into Y: component q of group G goes to head q / fold, frequency G*fold + q % fold, the real and the
+ *     imaginary rows with the same U_G [g*fold, g*fold] (U [d/2/fold, g*fold, g*fold]).  Y must not alias X.
+ *   transmla_conv_alpha: Eq. 19, *alpha_out (device) = mean_t ||k_nope,t|| / mean_t ||v_t|| over the rows of
+ *     k_nope [n, mk] and v [n, mv]; scratch: 2n floats.  Deterministic summation order.
+ *   transmla_conv_balance_concat: Z [n, mk+mv] = [k_nope / alpha | v] (App. D.2 step 1), alpha read on the device.
+ *   transmla_conv_top_subspace: App. D.2 step 2 for a second-moment matrix too large for Jacobi: an orthonormal
+ *     basis Q [m, r] of the r leading eigenvectors' span of the symmetric positive semi-definite Cmat [m, m], by
+ *     `iters` rounds of Q <- orth(Cmat Q) (Cholesky QR applied twice, Gram matrix and factor in fp64).  Q holds the
+ *     start basis on entry (full column rank, e.g. random numbers drawn by the caller).  Any orthonormal basis of
+ *     the span gives the same converted layer (App. D.2: the latent may be re-based).  scratch: 256-byte aligned,
+ *     transmla_conv_subspace_scratch_bytes(m, r). */
+transmla_status_t transmla_conv_gemm(int ta, int tb, int M, int N, int K, float alpha, const float* A, int lda,
+                                     const float* B, int ldb, float* C, int ldc, void* stream);
+size_t transmla_conv_rorope_scratch_bytes(int n, int g, int d, int fold);
+transmla_status_t transmla_conv_rorope_covariance(const float* K, int n, int g, int d, int fold, void* scratch,
+                                                  size_t scratch_bytes, float* cov, void* stream);
+transmla_status_t transmla_conv_sym_eig(float* a, int batch, int m, float* eigvals, float* eigvecs, int32_t* dev_status,
+                                        void* stream);
+transmla_status_t transmla_conv_rorope_apply(const float* X, int C, const float* U, int g, int d, int fold, float* Y,
+                                             void* stream);
+transmla_status_t transmla_conv_alpha(const float* k_nope, int n, int mk, const float* v, int mv, float* scratch,
+                                      float* alpha_out, void* stream);
+transmla_status_t transmla_conv_balance_concat(const float* k_nope, int n, int mk, const float* v, int mv,
+                                               const float* alpha, float* Z, void* stream);
+size_t transmla_conv_subspace_scratch_bytes(int m, int r);
+transmla_status_t transmla_conv_top_subspace(const float* Cmat, int m, int r, int iters, float* Q, void* scratch,
+                                             size_t scratch_bytes, int32_t* dev_status, void* stream);
 
 /* Whether transmla_mla_decode with these `params` hands pages to CTAs at run time (1) or keeps to the page ranges of
  * the split plan (0); see transmla_params_t.num_partitions.  With run-time claims the default path is not

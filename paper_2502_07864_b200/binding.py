@@ -17,7 +17,10 @@ EXPORTS = ('transmla_workspace_layout', 'transmla_latent_append', 'transmla_mla_
            'transmla_static_workspace_capacity', 'transmla_mla_attention_static', 'transmla_selftest_bounded_wait',
            'transmla_layer_scratch_bytes', 'transmla_layer_decode_step', 'transmla_stream_probe', 'transmla_page_claims_at_run_time', 'transmla_latent_append_fp8',
            'transmla_mla_decode_fp8', 'transmla_prefill_scratch_bytes', 'transmla_prefill_decompress',
-           'transmla_prefill_attention', 'transmla_mla_prefill')
+           'transmla_prefill_attention', 'transmla_mla_prefill', 'transmla_conv_gemm',
+           'transmla_conv_rorope_scratch_bytes', 'transmla_conv_rorope_covariance', 'transmla_conv_sym_eig',
+           'transmla_conv_rorope_apply', 'transmla_conv_alpha', 'transmla_conv_balance_concat',
+           'transmla_conv_subspace_scratch_bytes', 'transmla_conv_top_subspace')
 
 
 class Params(ctypes.Structure):
@@ -83,6 +86,18 @@ def lib():
         L.transmla_prefill_decompress.argtypes = [pp, vp, i32p, i32p, vp, vp, vp, sz, i32p, vp]
         L.transmla_prefill_attention.argtypes = [pp, vp, vp, vp, vp, sz, i32p, i32p, vp, vp, i32p, vp]
         L.transmla_mla_prefill.argtypes = [pp, vp, vp, vp, vp, vp, i32p, i32p, vp, sz, vp, vp, i32p, vp]
+        ci, cf = ctypes.c_int, ctypes.c_float
+        L.transmla_conv_gemm.argtypes = [ci, ci, ci, ci, ci, cf, vp, ci, vp, ci, vp, ci, vp]
+        L.transmla_conv_rorope_scratch_bytes.argtypes = [ci, ci, ci, ci]
+        L.transmla_conv_rorope_scratch_bytes.restype = sz
+        L.transmla_conv_rorope_covariance.argtypes = [vp, ci, ci, ci, ci, vp, sz, vp, vp]
+        L.transmla_conv_sym_eig.argtypes = [vp, ci, ci, vp, vp, i32p, vp]
+        L.transmla_conv_rorope_apply.argtypes = [vp, ci, vp, ci, ci, ci, vp, vp]
+        L.transmla_conv_alpha.argtypes = [vp, ci, ci, vp, ci, vp, vp, vp]
+        L.transmla_conv_balance_concat.argtypes = [vp, ci, ci, vp, ci, vp, vp, vp]
+        L.transmla_conv_subspace_scratch_bytes.argtypes = [ci, ci]
+        L.transmla_conv_subspace_scratch_bytes.restype = sz
+        L.transmla_conv_top_subspace.argtypes = [vp, ci, ci, ci, vp, vp, sz, i32p, vp]
         L.transmla_layer_scratch_bytes.argtypes = [pp, ctypes.c_int32]
         L.transmla_layer_scratch_bytes.restype = sz
         L.transmla_layer_decode_step.argtypes = [pp, ctypes.POINTER(LayerWeights), vp, i32p, i32p, vp, vp, sz, vp, sz, vp,
@@ -263,6 +278,55 @@ def transmla_mla_prefill(params, q_nope, q_pe, w_uk, w_uv, cache, page_table, se
                                       _ptr(page_table), _ptr(seqlens), _ptr(scratch), _nbytes(scratch), _ptr(out), _ptr(lse),
                                       _ptr(dev_status), _stream(stream)),
            'transmla_mla_prefill')
+
+
+# ---- conversion calls: fp32 device tensors, row-major and contiguous
+def transmla_conv_gemm(a, b, c, ta=False, tb=False, alpha=1.0, stream=None):
+    """c[M,N] = alpha * op(a) op(b); shapes are taken from the tensors."""
+    M, N = c.shape
+    K = a.shape[0] if ta else a.shape[1]
+    _check(lib().transmla_conv_gemm(int(ta), int(tb), M, N, K, float(alpha), _ptr(a), a.shape[1], _ptr(b), b.shape[1],
+                                    _ptr(c), c.shape[1], _stream(stream)), 'transmla_conv_gemm')
+
+
+def transmla_conv_rorope_covariance(k_act, g, d, fold, scratch, cov, stream=None):
+    _check(lib().transmla_conv_rorope_covariance(_ptr(k_act), k_act.shape[0], g, d, fold, _ptr(scratch), _nbytes(scratch),
+                                                 _ptr(cov), _stream(stream)), 'transmla_conv_rorope_covariance')
+
+
+def transmla_conv_rorope_scratch_bytes(n, g, d, fold):
+    return int(lib().transmla_conv_rorope_scratch_bytes(n, g, d, fold))
+
+
+def transmla_conv_sym_eig(a, eigvals, eigvecs, dev_status=None, stream=None):
+    batch, m, _ = a.shape
+    _check(lib().transmla_conv_sym_eig(_ptr(a), batch, m, _ptr(eigvals), _ptr(eigvecs), _ptr(dev_status), _stream(stream)),
+           'transmla_conv_sym_eig')
+
+
+def transmla_conv_rorope_apply(x, u, g, d, fold, y, stream=None):
+    _check(lib().transmla_conv_rorope_apply(_ptr(x), x.shape[1], _ptr(u), g, d, fold, _ptr(y), _stream(stream)),
+           'transmla_conv_rorope_apply')
+
+
+def transmla_conv_alpha(k_nope, v, scratch, alpha_out, stream=None):
+    _check(lib().transmla_conv_alpha(_ptr(k_nope), k_nope.shape[0], k_nope.shape[1], _ptr(v), v.shape[1], _ptr(scratch),
+                                     _ptr(alpha_out), _stream(stream)), 'transmla_conv_alpha')
+
+
+def transmla_conv_balance_concat(k_nope, v, alpha, z, stream=None):
+    _check(lib().transmla_conv_balance_concat(_ptr(k_nope), k_nope.shape[0], k_nope.shape[1], _ptr(v), v.shape[1], _ptr(alpha),
+                                              _ptr(z), _stream(stream)), 'transmla_conv_balance_concat')
+
+
+def transmla_conv_subspace_scratch_bytes(m, r):
+    return int(lib().transmla_conv_subspace_scratch_bytes(m, r))
+
+
+def transmla_conv_top_subspace(cmat, q, iters, scratch, dev_status=None, stream=None):
+    m, r = q.shape
+    _check(lib().transmla_conv_top_subspace(_ptr(cmat), m, r, iters, _ptr(q), _ptr(scratch), _nbytes(scratch), _ptr(dev_status),
+                                            _stream(stream)), 'transmla_conv_top_subspace')
 
 
 def transmla_page_claims_at_run_time(params):

@@ -7,7 +7,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, 'csrc')
 LIB = os.path.join(HERE, 'libtransmla.so')
-SOURCES = ['api.cu', 'small_kernels.cu', 'decode_generic.cu', 'decode_sm100.cu', 'static_workspace.cu', 'selftest.cu', 'linear.cu', 'linear_sm100.cu', 'stream_probe.cu', 'decode_fp8.cu', 'append_fp8.cu', 'prefill_decompress.cu', 'prefill_attention.cu', 'prefill_api.cu']
+SOURCES = ['api.cu', 'small_kernels.cu', 'decode_generic.cu', 'decode_sm100.cu', 'static_workspace.cu', 'selftest.cu', 'linear.cu', 'linear_sm100.cu', 'stream_probe.cu', 'decode_fp8.cu', 'append_fp8.cu', 'prefill_decompress.cu', 'prefill_attention.cu', 'prefill_api.cu', 'conversion.cu', 'conversion_api.cu']
 
 
 def _stale():

@@ -1,0 +1,361 @@
+// Kernels of the GQA -> MLA conversion on calibration activations (Sec. 4.2, 4.3; App. B, C, D).
+// fp32 SIMT arithmetic (fp64 where the orthonormalisation needs it): the results are eigenvectors and low-rank
+// bases, and the step is a one-off per model, bound by the two large contractions (the joint second moment and
+// the subspace iteration's products).
+#include "conversion.cuh"
+
+namespace transmla {
+namespace conv {
+
+// ------------------------------------------------------------------------------------------------ GEMM
+// 128 x 128 tile, 256 threads x (8 x 8) outputs, k in steps of 8 through shared memory.  Any of the four
+// storage combinations; edges are bounds-checked, so no shape restriction.
+constexpr int BM = 128, BN = 128, BK = 8;
+
+template <typename TOut>
+__global__ void __launch_bounds__(256) gemm_kernel(int ta, int tb, int M, int N, int K, float alpha, const float* A, int lda,
+                                                   long long strideA, const float* B, int ldb, long long strideB, TOut* C,
+                                                   int ldc, long long strideC) {
+  __shared__ float As[BK][BM + 4];
+  __shared__ float Bs[BK][BN + 4];
+  A += strideA * blockIdx.z;
+  B += strideB * blockIdx.z;
+  C += strideC * blockIdx.z;
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  TOut acc[8][8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[i][j] = TOut(0);
+  for (int k0 = 0; k0 < K; k0 += BK) {
+    // tile loads: walk the contiguous storage dimension with consecutive threads
+    for (int e = tid; e < BM * BK; e += 256) {
+      int mm, kk;
+      if (ta) { mm = e % BM; kk = e / BM; } else { kk = e % BK; mm = e / BK; }
+      const int m = m0 + mm, k = k0 + kk;
+      float v = 0.f;
+      if (m < M && k < K) v = ta ? A[static_cast<size_t>(k) * lda + m] : A[static_cast<size_t>(m) * lda + k];
+      As[kk][mm] = v;
+    }
+    for (int e = tid; e < BN * BK; e += 256) {
+      int nn, kk;
+      if (tb) { kk = e % BK; nn = e / BK; } else { nn = e % BN; kk = e / BN; }
+      const int n = n0 + nn, k = k0 + kk;
+      float v = 0.f;
+      if (n < N && k < K) v = tb ? B[static_cast<size_t>(n) * ldb + k] : B[static_cast<size_t>(k) * ldb + n];
+      Bs[kk][nn] = v;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < BK; ++kk) {
+      float a[8], b[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) a[i] = As[kk][ty * 4 + (i & 3) + (i >> 2) * 64];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) b[j] = Bs[kk][tx * 4 + (j & 3) + (j >> 2) * 64];
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[i][j] += static_cast<TOut>(a[i]) * static_cast<TOut>(b[j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int m = m0 + ty * 4 + (i & 3) + (i >> 2) * 64;
+    if (m >= M) continue;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int n = n0 + tx * 4 + (j & 3) + (j >> 2) * 64;
+      if (n < N) C[static_cast<size_t>(m) * ldc + n] = static_cast<TOut>(alpha) * acc[i][j];
+    }
+  }
+}
+
+cudaError_t gemm_f32(int ta, int tb, int M, int N, int K, float alpha, const float* A, int lda, long long strideA,
+                     const float* B, int ldb, long long strideB, float* C, int ldc, long long strideC, int batch,
+                     cudaStream_t stream) {
+  if (M <= 0 || N <= 0 || batch <= 0) return cudaSuccess;
+  dim3 grid((N + BN - 1) / BN, (M + BM - 1) / BM, batch);
+  gemm_kernel<float><<<grid, 256, 0, stream>>>(ta, tb, M, N, K, alpha, A, lda, strideA, B, ldb, strideB, C, ldc, strideC);
+  return cudaGetLastError();
+}
+
+cudaError_t gemm_f32_to_f64(int ta, int tb, int M, int N, int K, const float* A, int lda, const float* B, int ldb, double* C,
+                            int ldc, cudaStream_t stream) {
+  if (M <= 0 || N <= 0) return cudaSuccess;
+  dim3 grid((N + BN - 1) / BN, (M + BM - 1) / BM, 1);
+  gemm_kernel<double><<<grid, 256, 0, stream>>>(ta, tb, M, N, K, 1.f, A, lda, 0, B, ldb, 0, C, ldc, 0);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------ RoRoPE helpers
+// Position in the merged key of segment entry i of group G (i = p*g + j: frequency G*fold + p, head j), real part.
+__device__ __forceinline__ int seg_pos(int G, int i, int g, int d, int fold) {
+  const int p = i / g, j = i - p * g;
+  return j * d + 2 * (G * fold + p);
+}
+
+__global__ void gather_segments_kernel(const float* K, int n, int g, int d, int fold, float* seg) {
+  const int m = g * fold, G = blockIdx.y;
+  const size_t total = static_cast<size_t>(2) * n * m;
+  for (size_t e = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; e < total; e += static_cast<size_t>(gridDim.x) * blockDim.x) {
+    const int i = static_cast<int>(e % m);
+    const size_t row = e / m;                       // 0..2n-1
+    const int t = static_cast<int>(row % n), im = static_cast<int>(row / n);
+    seg[static_cast<size_t>(G) * total + e] = K[static_cast<size_t>(t) * g * d + seg_pos(G, i, g, d, fold) + im];
+  }
+}
+
+cudaError_t gather_segments(const float* K, int n, int g, int d, int fold, float* seg, cudaStream_t stream) {
+  const int groups = d / 2 / fold;
+  dim3 grid(296, groups);
+  gather_segments_kernel<<<grid, 256, 0, stream>>>(K, n, g, d, fold, seg);
+  return cudaGetLastError();
+}
+
+// Y[(q / fold, 2 (G fold + q % fold) + im), c] = sum_i U_G[i, q] X[seg_pos(G, i) + im, c]   (Eq. 18)
+__global__ void rorope_apply_kernel(const float* X, int C, const float* U, int g, int d, int fold, float* Y) {
+  const int m = g * fold, G = blockIdx.y, im = blockIdx.z;
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  extern __shared__ float u_s[];  // U_G [m][m]
+  for (int e = threadIdx.x; e < m * m; e += blockDim.x) u_s[e] = U[static_cast<size_t>(G) * m * m + e];
+  __syncthreads();
+  if (c >= C) return;
+  for (int q0 = 0; q0 < m; q0 += 8) {
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    for (int i = 0; i < m; ++i) {
+      const float x = X[static_cast<size_t>(seg_pos(G, i, g, d, fold) + im) * C + c];
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        if (q0 + u < m) acc[u] = fmaf(u_s[i * m + q0 + u], x, acc[u]);
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int q = q0 + u;
+      if (q < m) Y[static_cast<size_t>((q / fold) * d + 2 * (G * fold + q % fold) + im) * C + c] = acc[u];
+    }
+  }
+}
+
+cudaError_t rorope_apply(const float* X, int C, const float* U, int g, int d, int fold, float* Y, cudaStream_t stream) {
+  const int m = g * fold, groups = d / 2 / fold;
+  const size_t smem = static_cast<size_t>(m) * m * sizeof(float);
+  if (smem > 48 * 1024) {
+    if (cudaError_t e = cudaFuncSetAttribute(rorope_apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+        e != cudaSuccess)
+      return e;
+  }
+  dim3 grid((C + 127) / 128, groups, 2);
+  rorope_apply_kernel<<<grid, 128, smem, stream>>>(X, C, U, g, d, fold, Y);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------ Eq. 19
+// norms[0..n) = ||k_nope,t||, norms[n..2n) = ||v_t||: one warp per row; then one block sums both halves in a fixed
+// order (the same bits on every run) and writes alpha = mean ||k|| / mean ||v||.
+__global__ void row_norms_kernel(const float* a, int n, int m, float* out) {
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (row >= n) return;
+  float s = 0.f;
+  for (int c = lane; c < m; c += 32) { const float x = a[static_cast<size_t>(row) * m + c]; s = fmaf(x, x, s); }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  if (lane == 0) out[row] = sqrtf(s);
+}
+__global__ void __launch_bounds__(1024) alpha_kernel(const float* norms, int n, float* alpha_out) {
+  __shared__ double part[2][1024];
+  double sk = 0.0, sv = 0.0;
+  for (int i = threadIdx.x; i < n; i += 1024) { sk += norms[i]; sv += norms[n + i]; }
+  part[0][threadIdx.x] = sk; part[1][threadIdx.x] = sv;
+  __syncthreads();
+  for (int o = 512; o > 0; o >>= 1) {
+    if (threadIdx.x < o) { part[0][threadIdx.x] += part[0][threadIdx.x + o]; part[1][threadIdx.x] += part[1][threadIdx.x + o]; }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) *alpha_out = static_cast<float>(part[0][0] / part[1][0]);
+}
+cudaError_t row_norm_ratio(const float* k_nope, int n, int mk, const float* v, int mv, float* scratch, float* alpha_out,
+                           cudaStream_t stream) {
+  row_norms_kernel<<<(n + 7) / 8, 256, 0, stream>>>(k_nope, n, mk, scratch);
+  row_norms_kernel<<<(n + 7) / 8, 256, 0, stream>>>(v, n, mv, scratch + n);
+  alpha_kernel<<<1, 1024, 0, stream>>>(scratch, n, alpha_out);
+  return cudaGetLastError();
+}
+
+// Z[t] = [k_nope,t / alpha ; v_t]   (App. D.2 step 1)
+__global__ void balance_concat_kernel(const float* k_nope, int n, int mk, const float* v, int mv, const float* alpha, float* Z) {
+  const float inv = 1.f / *alpha;
+  const int m = mk + mv;
+  const size_t total = static_cast<size_t>(n) * m;
+  for (size_t e = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; e < total; e += static_cast<size_t>(gridDim.x) * blockDim.x) {
+    const size_t t = e / m;
+    const int c = static_cast<int>(e % m);
+    Z[e] = c < mk ? k_nope[t * mk + c] * inv : v[t * mv + (c - mk)];
+  }
+}
+cudaError_t balance_concat(const float* k_nope, int n, int mk, const float* v, int mv, const float* alpha, float* Z,
+                           cudaStream_t stream) {
+  balance_concat_kernel<<<592, 256, 0, stream>>>(k_nope, n, mk, v, mv, alpha, Z);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------ eigenvectors
+// Parallel cyclic Jacobi for a symmetric matrix of order m <= 128, one block per matrix, A and V in shared memory.
+// A round rotates m/2 disjoint index pairs (round-robin tournament), all with angles taken from the matrix as it
+// stands before the round: columns first (A <- A J, V <- V J), then rows (A <- J^T A).  Sweeps stop when the
+// off-diagonal mass is below fp32 resolution of the whole; the eigenvalues are then sorted in descending order.
+constexpr int kEigMax = 128, kEigSweeps = 30;
+
+__global__ void __launch_bounds__(256) jacobi_eigh_kernel(const float* a_in, int m, float* eigvals, float* eigvecs,
+                                                          int32_t* dev_status) {
+  extern __shared__ float es[];
+  const int ld = m + 1, mm = (m + 1) & ~1, half = mm / 2;
+  float* A = es;                    // [m][ld]
+  float* V = A + m * ld;            // [m][ld]
+  float* cs = V + m * ld;           // [half][2]
+  int* pq = reinterpret_cast<int*>(cs + 2 * half);  // [half][2]
+  int* order = pq + 2 * half;       // [m]
+  __shared__ float red[256];
+  __shared__ int done;
+  const int tid = threadIdx.x;
+  const float* src = a_in + static_cast<size_t>(blockIdx.x) * m * m;
+  for (int e = tid; e < m * m; e += 256) {
+    const int i = e / m, j = e % m;
+    A[i * ld + j] = 0.5f * (src[e] + src[j * m + i]);  // exactly symmetric whatever rounding the input carries
+    V[i * ld + j] = i == j ? 1.f : 0.f;
+  }
+  if (tid == 0) done = 0;
+  __syncthreads();
+  for (int sweep = 0; sweep < kEigSweeps; ++sweep) {
+    // convergence: off-diagonal sum of squares against the whole
+    float off = 0.f, tot = 0.f;
+    for (int e = tid; e < m * m; e += 256) {
+      const int i = e / m, j = e % m;
+      const float x = A[i * ld + j];
+      tot += x * x;
+      if (i != j) off += x * x;
+    }
+    red[tid] = off; __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) { if (tid < o) red[tid] += red[tid + o]; __syncthreads(); }
+    const float off_all = red[0]; __syncthreads();
+    red[tid] = tot; __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) { if (tid < o) red[tid] += red[tid + o]; __syncthreads(); }
+    const float tot_all = red[0]; __syncthreads();
+    if (off_all <= 1e-13f * tot_all) { if (tid == 0) done = 1; __syncthreads(); break; }
+    for (int rd = 0; rd < mm - 1; ++rd) {
+      if (tid < half) {
+        int p, q;
+        if (tid == 0) { p = mm - 1; q = rd; }
+        else { p = (rd + tid) % (mm - 1); q = (rd - tid + mm - 1) % (mm - 1); }
+        if (p > q) { const int t = p; p = q; q = t; }
+        float c = 1.f, s = 0.f;
+        if (q < m) {
+          const float apq = A[p * ld + q], app = A[p * ld + p], aqq = A[q * ld + q];
+          if (fabsf(apq) > 1e-30f) {
+            const float theta = (aqq - app) / (2.f * apq);
+            const float t = (theta >= 0.f ? 1.f : -1.f) / (fabsf(theta) + sqrtf(theta * theta + 1.f));
+            c = 1.f / sqrtf(t * t + 1.f);
+            s = t * c;
+          }
+        } else { p = -1; }
+        pq[2 * tid] = p; pq[2 * tid + 1] = q; cs[2 * tid] = c; cs[2 * tid + 1] = s;
+      }
+      __syncthreads();
+      for (int e = tid; e < half * m; e += 256) {      // columns p, q of A and V
+        const int k = e / m, i = e % m, p = pq[2 * k], q = pq[2 * k + 1];
+        if (p < 0) continue;
+        const float c = cs[2 * k], s = cs[2 * k + 1];
+        const float ap = A[i * ld + p], aq = A[i * ld + q];
+        A[i * ld + p] = c * ap - s * aq; A[i * ld + q] = s * ap + c * aq;
+        const float vp = V[i * ld + p], vq = V[i * ld + q];
+        V[i * ld + p] = c * vp - s * vq; V[i * ld + q] = s * vp + c * vq;
+      }
+      __syncthreads();
+      for (int e = tid; e < half * m; e += 256) {      // rows p, q of A
+        const int k = e / m, j = e % m, p = pq[2 * k], q = pq[2 * k + 1];
+        if (p < 0) continue;
+        const float c = cs[2 * k], s = cs[2 * k + 1];
+        const float ap = A[p * ld + j], aq = A[q * ld + j];
+        A[p * ld + j] = c * ap - s * aq; A[q * ld + j] = s * ap + c * aq;
+      }
+      __syncthreads();
+    }
+  }
+  if (tid == 0) {
+    if (!done && dev_status != nullptr) atomicOr(dev_status, TRANSMLA_DEV_NUMERIC);
+    for (int i = 0; i < m; ++i) order[i] = i;
+    for (int i = 0; i < m; ++i) {       // selection sort, descending (stable for equal values)
+      int best = i;
+      for (int j = i + 1; j < m; ++j)
+        if (A[order[j] * ld + order[j]] > A[order[best] * ld + order[best]]) best = j;
+      const int t = order[best];
+      for (int j = best; j > i; --j) order[j] = order[j - 1];
+      order[i] = t;
+    }
+  }
+  __syncthreads();
+  float* w = eigvals + static_cast<size_t>(blockIdx.x) * m;
+  float* vec = eigvecs + static_cast<size_t>(blockIdx.x) * m * m;
+  for (int q = tid; q < m; q += 256) w[q] = A[order[q] * ld + order[q]];
+  for (int e = tid; e < m * m; e += 256) { const int i = e / m, q = e % m; vec[e] = V[i * ld + order[q]]; }
+}
+
+cudaError_t sym_eig(float* a, int batch, int m, float* eigvals, float* eigvecs, int32_t* dev_status, cudaStream_t stream) {
+  if (m < 1 || m > kEigMax) return cudaErrorInvalidValue;
+  const int half = ((m + 1) & ~1) / 2;
+  const size_t smem = (static_cast<size_t>(2) * m * (m + 1) + 4 * half + m) * sizeof(float);
+  if (cudaError_t e = cudaFuncSetAttribute(jacobi_eigh_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+      e != cudaSuccess)
+    return e;
+  jacobi_eigh_kernel<<<batch, 256, smem, stream>>>(a, m, eigvals, eigvecs, dev_status);
+  return cudaGetLastError();
+}
+// ------------------------------------------------------------------------------------------------ orthonormalisation
+// G = L L^T (fp64, in place in the lower triangle), then Linv = L^-1 (lower triangular, written as fp32 with zeros
+// above the diagonal).  One block; r up to a few hundred, r^3 / 3 operations twice.
+__global__ void __launch_bounds__(1024) cholesky_inverse_kernel(double* G, int r, double* Lw, float* Linv, int32_t* dev_status) {
+  const int tid = threadIdx.x;
+  __shared__ int bad;
+  if (tid == 0) bad = 0;
+  __syncthreads();
+  for (int k = 0; k < r; ++k) {
+    if (tid == 0) {
+      const double d = G[static_cast<size_t>(k) * r + k];
+      if (!(d > 0.0)) { bad = 1; G[static_cast<size_t>(k) * r + k] = 1.0; }
+      else G[static_cast<size_t>(k) * r + k] = sqrt(d);
+    }
+    __syncthreads();
+    const double dk = G[static_cast<size_t>(k) * r + k];
+    for (int i = k + 1 + tid; i < r; i += 1024) G[static_cast<size_t>(i) * r + k] /= dk;
+    __syncthreads();
+    const int rem = r - k - 1;
+    for (long long e = tid; e < static_cast<long long>(rem) * rem; e += 1024) {
+      const int i = k + 1 + static_cast<int>(e / rem), j = k + 1 + static_cast<int>(e % rem);
+      if (j <= i) G[static_cast<size_t>(i) * r + j] -= G[static_cast<size_t>(i) * r + k] * G[static_cast<size_t>(j) * r + k];
+    }
+    __syncthreads();
+  }
+  // inverse of the lower-triangular factor, column by column: X[j][j] = 1/L[j][j]; X[i][j] = -sum_{k=j}^{i-1} L[i][k] X[k][j] / L[i][i]
+  for (int j = tid; j < r; j += 1024) {
+    for (int i = 0; i < r; ++i) Lw[static_cast<size_t>(i) * r + j] = 0.0;
+    Lw[static_cast<size_t>(j) * r + j] = 1.0 / G[static_cast<size_t>(j) * r + j];
+    for (int i = j + 1; i < r; ++i) {
+      double s = 0.0;
+      for (int k = j; k < i; ++k) s += G[static_cast<size_t>(i) * r + k] * Lw[static_cast<size_t>(k) * r + j];
+      Lw[static_cast<size_t>(i) * r + j] = -s / G[static_cast<size_t>(i) * r + i];
+    }
+  }
+  __syncthreads();
+  for (long long e = tid; e < static_cast<long long>(r) * r; e += 1024) Linv[e] = static_cast<float>(Lw[e]);
+  if (tid == 0 && bad && dev_status != nullptr) atomicOr(dev_status, TRANSMLA_DEV_NUMERIC);
+}
+
+cudaError_t cholesky_inverse(double* G, int r, double* work, float* Linv, int32_t* dev_status, cudaStream_t stream) {
+  cholesky_inverse_kernel<<<1, 1024, 0, stream>>>(G, r, work, Linv, dev_status);
+  return cudaGetLastError();
+}
+
+}  // namespace conv
+}  // namespace transmla

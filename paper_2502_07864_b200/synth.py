@@ -149,3 +149,16 @@ def make_layer_weights(shape, seed, q_lora_rank=0, device='cpu'):
     if q_lora_rank:
         w['w_dq'] = _randn_bf16((q_lora_rank, shape.D), shape.D ** -0.5, g, device)
     return w
+
+
+def make_conversion_case(n, D, g, d, seed, device='cpu', key_gain=3.0):
+    """Calibration inputs of the conversion (Sec. 4.2, 4.3), fp32: hidden states x [n, D] whose coordinates decay like
+    i**-0.5 (a few strong directions, as the hidden states of a trained model have), key and value projections
+    w_k, w_v [g*d, D] ~ N(0, 1/sqrt(D)) with the keys `key_gain` times larger (the imbalance Eq. 19 is there for), and
+    a start basis for the subspace iteration is left to the caller.  No arithmetic of the method happens here."""
+    gen = _gen(seed, device)
+    scale = torch.arange(1, D + 1, dtype=torch.float32, device=device) ** -0.5
+    x = torch.randn(n, D, generator=gen, device=device) * scale * (D ** 0.5 / scale.norm())
+    w_k = torch.randn(g * d, D, generator=gen, device=device) * (key_gain * D ** -0.5)
+    w_v = torch.randn(g * d, D, generator=gen, device=device) * D ** -0.5
+    return {'x': x, 'w_k': w_k, 'w_v': w_v}
