@@ -375,7 +375,8 @@ transmla_status_t transmla_mla_prefill(const transmla_params_t* params /* host *
  *   transmla_conv_balance_concat: Z [n, mk+mv] = [k_nope / alpha | v] (App. D.2 step 1), alpha read on the device.
  *   transmla_conv_top_subspace: App. D.2 step 2 for a second-moment matrix too large for Jacobi: an orthonormal
  *     basis Q [m, r] of the r leading eigenvectors' span of the symmetric positive semi-definite Cmat [m, m], by
- *     `iters` rounds of Q <- orth(Cmat Q) (Cholesky QR applied twice, Gram matrix and factor in fp64).  Q holds the
+ *     `iters` rounds of Q <- orth(Cmat Q) (Cholesky QR with the Gram matrix and its factor in fp64: one per round,
+ *     two before the first round and one more after the last; r <= 1024).  Q holds the
  *     start basis on entry (full column rank, e.g. random numbers drawn by the caller).  Any orthonormal basis of
  *     the span gives the same converted layer (App. D.2: the latent may be re-based).  scratch: 256-byte aligned,
  *     transmla_conv_subspace_scratch_bytes(m, r). */

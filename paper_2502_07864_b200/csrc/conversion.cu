@@ -206,9 +206,9 @@ cudaError_t balance_concat(const float* k_nope, int n, int mk, const float* v, i
 // A round rotates m/2 disjoint index pairs (round-robin tournament), all with angles taken from the matrix as it
 // stands before the round: columns first (A <- A J, V <- V J), then rows (A <- J^T A).  Sweeps stop when the
 // off-diagonal mass is below fp32 resolution of the whole; the eigenvalues are then sorted in descending order.
-constexpr int kEigMax = 128, kEigSweeps = 30;
+constexpr int kEigMax = 128, kEigSweeps = 30, kEigThreads = 512;
 
-__global__ void __launch_bounds__(256) jacobi_eigh_kernel(const float* a_in, int m, float* eigvals, float* eigvecs,
+__global__ void __launch_bounds__(kEigThreads) jacobi_eigh_kernel(const float* a_in, int m, float* eigvals, float* eigvecs,
                                                           int32_t* dev_status) {
   extern __shared__ float es[];
   const int ld = m + 1, mm = (m + 1) & ~1, half = mm / 2;
@@ -217,33 +217,41 @@ __global__ void __launch_bounds__(256) jacobi_eigh_kernel(const float* a_in, int
   float* cs = V + m * ld;           // [half][2]
   int* pq = reinterpret_cast<int*>(cs + 2 * half);  // [half][2]
   int* order = pq + 2 * half;       // [m]
-  __shared__ float red[256];
+  __shared__ float red[kEigThreads];
   __shared__ int done;
   const int tid = threadIdx.x;
   const float* src = a_in + static_cast<size_t>(blockIdx.x) * m * m;
-  for (int e = tid; e < m * m; e += 256) {
+  for (int e = tid; e < m * m; e += kEigThreads) {
     const int i = e / m, j = e % m;
     A[i * ld + j] = 0.5f * (src[e] + src[j * m + i]);  // exactly symmetric whatever rounding the input carries
     V[i * ld + j] = i == j ? 1.f : 0.f;
   }
   if (tid == 0) done = 0;
   __syncthreads();
+  float prev_off = 3.4e38f;
   for (int sweep = 0; sweep < kEigSweeps; ++sweep) {
     // convergence: off-diagonal sum of squares against the whole
     float off = 0.f, tot = 0.f;
-    for (int e = tid; e < m * m; e += 256) {
+    for (int e = tid; e < m * m; e += kEigThreads) {
       const int i = e / m, j = e % m;
       const float x = A[i * ld + j];
       tot += x * x;
       if (i != j) off += x * x;
     }
     red[tid] = off; __syncthreads();
-    for (int o = 128; o > 0; o >>= 1) { if (tid < o) red[tid] += red[tid + o]; __syncthreads(); }
+    for (int o = kEigThreads / 2; o > 0; o >>= 1) { if (tid < o) red[tid] += red[tid + o]; __syncthreads(); }
     const float off_all = red[0]; __syncthreads();
     red[tid] = tot; __syncthreads();
-    for (int o = 128; o > 0; o >>= 1) { if (tid < o) red[tid] += red[tid + o]; __syncthreads(); }
+    for (int o = kEigThreads / 2; o > 0; o >>= 1) { if (tid < o) red[tid] += red[tid + o]; __syncthreads(); }
     const float tot_all = red[0]; __syncthreads();
-    if (off_all <= 1e-13f * tot_all) { if (tid == 0) done = 1; __syncthreads(); break; }
+    // converged: the off-diagonal mass is gone, or it sits at the fp32 rounding floor of the rotations (it has
+    // stopped shrinking and is below 1e-8 of the whole)
+    if (off_all <= 1e-13f * tot_all || (sweep >= 4 && off_all > 0.25f * prev_off && off_all <= 1e-8f * tot_all)) {
+      if (tid == 0) done = 1;
+      __syncthreads();
+      break;
+    }
+    prev_off = off_all;
     for (int rd = 0; rd < mm - 1; ++rd) {
       if (tid < half) {
         int p, q;
@@ -263,7 +271,7 @@ __global__ void __launch_bounds__(256) jacobi_eigh_kernel(const float* a_in, int
         pq[2 * tid] = p; pq[2 * tid + 1] = q; cs[2 * tid] = c; cs[2 * tid + 1] = s;
       }
       __syncthreads();
-      for (int e = tid; e < half * m; e += 256) {      // columns p, q of A and V
+      for (int e = tid; e < half * m; e += kEigThreads) {      // columns p, q of A and V
         const int k = e / m, i = e % m, p = pq[2 * k], q = pq[2 * k + 1];
         if (p < 0) continue;
         const float c = cs[2 * k], s = cs[2 * k + 1];
@@ -273,7 +281,7 @@ __global__ void __launch_bounds__(256) jacobi_eigh_kernel(const float* a_in, int
         V[i * ld + p] = c * vp - s * vq; V[i * ld + q] = s * vp + c * vq;
       }
       __syncthreads();
-      for (int e = tid; e < half * m; e += 256) {      // rows p, q of A
+      for (int e = tid; e < half * m; e += kEigThreads) {      // rows p, q of A
         const int k = e / m, j = e % m, p = pq[2 * k], q = pq[2 * k + 1];
         if (p < 0) continue;
         const float c = cs[2 * k], s = cs[2 * k + 1];
@@ -298,8 +306,8 @@ __global__ void __launch_bounds__(256) jacobi_eigh_kernel(const float* a_in, int
   __syncthreads();
   float* w = eigvals + static_cast<size_t>(blockIdx.x) * m;
   float* vec = eigvecs + static_cast<size_t>(blockIdx.x) * m * m;
-  for (int q = tid; q < m; q += 256) w[q] = A[order[q] * ld + order[q]];
-  for (int e = tid; e < m * m; e += 256) { const int i = e / m, q = e % m; vec[e] = V[i * ld + order[q]]; }
+  for (int q = tid; q < m; q += kEigThreads) w[q] = A[order[q] * ld + order[q]];
+  for (int e = tid; e < m * m; e += kEigThreads) { const int i = e / m, q = e % m; vec[e] = V[i * ld + order[q]]; }
 }
 
 cudaError_t sym_eig(float* a, int batch, int m, float* eigvals, float* eigvecs, int32_t* dev_status, cudaStream_t stream) {
@@ -309,51 +317,77 @@ cudaError_t sym_eig(float* a, int batch, int m, float* eigvals, float* eigvecs, 
   if (cudaError_t e = cudaFuncSetAttribute(jacobi_eigh_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
       e != cudaSuccess)
     return e;
-  jacobi_eigh_kernel<<<batch, 256, smem, stream>>>(a, m, eigvals, eigvecs, dev_status);
+  jacobi_eigh_kernel<<<batch, kEigThreads, smem, stream>>>(a, m, eigvals, eigvecs, dev_status);
   return cudaGetLastError();
 }
 // ------------------------------------------------------------------------------------------------ orthonormalisation
-// G = L L^T (fp64, in place in the lower triangle), then Linv = L^-1 (lower triangular, written as fp32 with zeros
-// above the diagonal).  One block; r up to a few hundred, r^3 / 3 operations twice.
-__global__ void __launch_bounds__(1024) cholesky_inverse_kernel(double* G, int r, double* Lw, float* Linv, int32_t* dev_status) {
-  const int tid = threadIdx.x;
+// Cholesky QR: G = Y^T Y = L L^T, Q = Y L^-T.
+// cholesky_kernel: right-looking factorisation of the fp64 Gram matrix in place (one block, 32 x 32 threads over the
+// trailing block, the current column cached in shared memory); L is also written as fp32 for the solve.
+constexpr int kCholMax = 1024;
+__global__ void __launch_bounds__(1024) cholesky_kernel(double* G, int r, float* L32, int32_t* dev_status) {
+  __shared__ double col[kCholMax];
   __shared__ int bad;
+  const int tid = threadIdx.x, tx = tid & 31, ty = tid >> 5;
   if (tid == 0) bad = 0;
   __syncthreads();
   for (int k = 0; k < r; ++k) {
     if (tid == 0) {
-      const double d = G[static_cast<size_t>(k) * r + k];
-      if (!(d > 0.0)) { bad = 1; G[static_cast<size_t>(k) * r + k] = 1.0; }
-      else G[static_cast<size_t>(k) * r + k] = sqrt(d);
+      double d = G[static_cast<size_t>(k) * r + k];
+      if (!(d > 0.0)) { bad = 1; d = 1.0; }
+      col[k] = sqrt(d);
     }
     __syncthreads();
-    const double dk = G[static_cast<size_t>(k) * r + k];
-    for (int i = k + 1 + tid; i < r; i += 1024) G[static_cast<size_t>(i) * r + k] /= dk;
+    const double dk = col[k];
+    for (int i = k + 1 + tid; i < r; i += 1024) col[i] = G[static_cast<size_t>(i) * r + k] / dk;
     __syncthreads();
-    const int rem = r - k - 1;
-    for (long long e = tid; e < static_cast<long long>(rem) * rem; e += 1024) {
-      const int i = k + 1 + static_cast<int>(e / rem), j = k + 1 + static_cast<int>(e % rem);
-      if (j <= i) G[static_cast<size_t>(i) * r + j] -= G[static_cast<size_t>(i) * r + k] * G[static_cast<size_t>(j) * r + k];
+    for (int i = k + tid; i < r; i += 1024) {       // column k is final
+      G[static_cast<size_t>(i) * r + k] = col[i];
+      L32[static_cast<size_t>(i) * r + k] = static_cast<float>(col[i]);
+    }
+    for (int i = k + 1 + ty; i < r; i += 32) {      // trailing update, lower triangle only
+      const double li = col[i];
+      for (int j = k + 1 + tx; j <= i; j += 32) G[static_cast<size_t>(i) * r + j] -= li * col[j];
     }
     __syncthreads();
   }
-  // inverse of the lower-triangular factor, column by column: X[j][j] = 1/L[j][j]; X[i][j] = -sum_{k=j}^{i-1} L[i][k] X[k][j] / L[i][i]
-  for (int j = tid; j < r; j += 1024) {
-    for (int i = 0; i < r; ++i) Lw[static_cast<size_t>(i) * r + j] = 0.0;
-    Lw[static_cast<size_t>(j) * r + j] = 1.0 / G[static_cast<size_t>(j) * r + j];
-    for (int i = j + 1; i < r; ++i) {
-      double s = 0.0;
-      for (int k = j; k < i; ++k) s += G[static_cast<size_t>(i) * r + k] * Lw[static_cast<size_t>(k) * r + j];
-      Lw[static_cast<size_t>(i) * r + j] = -s / G[static_cast<size_t>(i) * r + i];
-    }
-  }
-  __syncthreads();
-  for (long long e = tid; e < static_cast<long long>(r) * r; e += 1024) Linv[e] = static_cast<float>(Lw[e]);
+  for (int e = tid; e < r * r; e += 1024) { if (e % r > e / r) L32[e] = 0.f; }
   if (tid == 0 && bad && dev_status != nullptr) atomicOr(dev_status, TRANSMLA_DEV_NUMERIC);
 }
 
-cudaError_t cholesky_inverse(double* G, int r, double* work, float* Linv, int32_t* dev_status, cudaStream_t stream) {
-  cholesky_inverse_kernel<<<1, 1024, 0, stream>>>(G, r, work, Linv, dev_status);
+// Q[row] L^T = Y[row]: forward substitution along the row, one warp per row (the dot product of step j is split
+// over the lanes), 8 rows per block kept in shared memory.  Q may alias Y.
+__global__ void __launch_bounds__(256) trsm_rows_kernel(const float* Y, int m, int r, const float* L32, float* Q) {
+  extern __shared__ float qs[];  // [8][r]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row = blockIdx.x * 8 + warp;
+  if (row >= m) return;
+  float* q = qs + warp * r;
+  for (int c = lane; c < r; c += 32) q[c] = Y[static_cast<size_t>(row) * r + c];
+  __syncwarp();
+  for (int j = 0; j < r; ++j) {
+    const float* lj = L32 + static_cast<size_t>(j) * r;
+    float s = 0.f;
+    for (int k = lane; k < j; k += 32) s = fmaf(q[k], lj[k], s);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) q[j] = (q[j] - s) / lj[j];
+    __syncwarp();
+  }
+  for (int c = lane; c < r; c += 32) Q[static_cast<size_t>(row) * r + c] = q[c];
+}
+
+cudaError_t cholesky_qr(const float* Y, int m, int r, double* G, float* L32, float* Q, int32_t* dev_status, cudaStream_t stream) {
+  if (r > kCholMax) return cudaErrorInvalidValue;
+  if (cudaError_t e = gemm_f32_to_f64(1, 0, r, r, m, Y, r, Y, r, G, r, stream); e != cudaSuccess) return e;
+  cholesky_kernel<<<1, 1024, 0, stream>>>(G, r, L32, dev_status);
+  const size_t smem = static_cast<size_t>(8) * r * sizeof(float);
+  if (smem > 48 * 1024) {
+    if (cudaError_t e = cudaFuncSetAttribute(trsm_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+        e != cudaSuccess)
+      return e;
+  }
+  trsm_rows_kernel<<<(m + 7) / 8, 256, smem, stream>>>(Y, m, r, L32, Q);
   return cudaGetLastError();
 }
 

@@ -26,9 +26,9 @@ cudaError_t row_norm_ratio(const float* k_nope, int n, int mk, const float* v, i
                            cudaStream_t stream);
 cudaError_t balance_concat(const float* k_nope, int n, int mk, const float* v, int mv, const float* alpha, float* Z,
                            cudaStream_t stream);
-// Cholesky factor of the fp64 Gram matrix G [r,r] (overwritten) and the inverse of the factor as fp32 Linv [r,r]
-// (lower triangular); work [r,r] fp64.  Sets TRANSMLA_DEV_NUMERIC if G is not positive definite.
-cudaError_t cholesky_inverse(double* G, int r, double* work, float* Linv, int32_t* dev_status, cudaStream_t stream);
+// Cholesky QR: Q [m,r] = Y L^-T with Y^T Y = L L^T (Gram matrix G [r,r] and its factor in fp64; L32 [r,r] the factor
+// in fp32 for the solve).  r <= 1024.  Q may alias Y.  Sets TRANSMLA_DEV_NUMERIC if the Gram matrix is not positive definite.
+cudaError_t cholesky_qr(const float* Y, int m, int r, double* G, float* L32, float* Q, int32_t* dev_status, cudaStream_t stream);
 
 }  // namespace conv
 }  // namespace transmla

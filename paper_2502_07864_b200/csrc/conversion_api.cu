@@ -68,36 +68,30 @@ transmla_status_t transmla_conv_balance_concat(const float* k_nope, int n, int m
 }
 
 size_t transmla_conv_subspace_scratch_bytes(int m, int r) {
-  if (m < 1 || r < 1 || r > m) return 0;
-  return static_cast<size_t>(m) * r * sizeof(float) + static_cast<size_t>(r) * r * (2 * sizeof(double) + sizeof(float)) + 512;
+  if (m < 1 || r < 1 || r > m || r > 1024) return 0;
+  return static_cast<size_t>(m) * r * sizeof(float) + static_cast<size_t>(r) * r * (sizeof(double) + sizeof(float)) + 512;
 }
 
 transmla_status_t transmla_conv_top_subspace(const float* Cmat, int m, int r, int iters, float* Q, void* scratch,
                                              size_t scratch_bytes, int32_t* dev_status, void* stream) {
   if (!Cmat || !Q || !scratch) return TRANSMLA_ERR_NULL;
-  if (m < 1 || r < 1 || r > m || iters < 1) return TRANSMLA_ERR_SHAPE;
+  if (m < 1 || r < 1 || r > m || r > 1024 || iters < 1) return TRANSMLA_ERR_SHAPE;
   if (!al16(Cmat) || !al16(Q) || (reinterpret_cast<uintptr_t>(scratch) & 255)) return TRANSMLA_ERR_ALIGN;
   if (scratch_bytes < transmla_conv_subspace_scratch_bytes(m, r)) return TRANSMLA_ERR_WORKSPACE;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   char* w = static_cast<char*>(scratch);
   double* G = reinterpret_cast<double*>(w);
-  double* Lw = G + static_cast<size_t>(r) * r;
-  float* Linv = reinterpret_cast<float*>(Lw + static_cast<size_t>(r) * r);
-  float* Y = reinterpret_cast<float*>(w + ((static_cast<size_t>(r) * r * (2 * sizeof(double) + sizeof(float)) + 255) & ~size_t(255)));
-  // Orthogonal iteration: Y = C Q, then Q = orth(Y) by Cholesky QR done twice (Gram matrix and factor in fp64).
-  auto orthonormalise = [&](float* src, float* dst) -> bool {   // dst = src L^-T with src^T src = L L^T
-    if (conv::gemm_f32_to_f64(1, 0, r, r, m, src, r, src, r, G, r, s) != cudaSuccess) return false;
-    if (conv::cholesky_inverse(G, r, Lw, Linv, dev_status, s) != cudaSuccess) return false;
-    return conv::gemm_f32(0, 1, m, r, r, 1.f, src, r, 0, Linv, r, 0, dst, r, 0, 1, s) == cudaSuccess;
-  };
-  if (!orthonormalise(Q, Y) || !orthonormalise(Y, Q)) return TRANSMLA_ERR_CUDA;
+  float* L32 = reinterpret_cast<float*>(G + static_cast<size_t>(r) * r);
+  float* Y = reinterpret_cast<float*>(w + ((static_cast<size_t>(r) * r * (sizeof(double) + sizeof(float)) + 255) & ~size_t(255)));
+  // Orthogonal iteration: Q <- orth(C Q).  One Cholesky QR per round keeps the columns independent; the basis is made
+  // orthonormal to fp32 resolution by the two passes at the start and the extra pass at the end.
+  auto orth = [&](float* y, float* q) { return conv::cholesky_qr(y, m, r, G, L32, q, dev_status, s) == cudaSuccess; };
+  if (!orth(Q, Q) || !orth(Q, Q)) return TRANSMLA_ERR_CUDA;
   for (int it = 0; it < iters; ++it) {
     if (conv::gemm_f32(0, 0, m, r, m, 1.f, Cmat, m, 0, Q, r, 0, Y, r, 0, 1, s) != cudaSuccess) return TRANSMLA_ERR_CUDA;
-    if (!orthonormalise(Y, Q) || !orthonormalise(Q, Y)) return TRANSMLA_ERR_CUDA;
-    if (cudaMemcpyAsync(Q, Y, static_cast<size_t>(m) * r * sizeof(float), cudaMemcpyDeviceToDevice, s) != cudaSuccess)
-      return TRANSMLA_ERR_CUDA;
+    if (!orth(Y, Q)) return TRANSMLA_ERR_CUDA;
   }
-  return TRANSMLA_OK;
+  return orth(Q, Q) ? TRANSMLA_OK : TRANSMLA_ERR_CUDA;
 }
 
 }  // extern "C"
