@@ -38,6 +38,8 @@ def workloads():
     w['qwen2.5-72b-mla_b64_s2'] = (synth.QWEN25_72B, synth.uniform_seqlens(64, 2048, 8192, 5), 5)
     for B in (16, 64, 128):      # the same shape over the FP8 latent cache (656 bytes a token instead of 1152)
         w[f'llama2-7b-mla-fp8_b{B}_8k'] = (synth.LLAMA2_7B, [8192] * B, 6)
+    # the conversion of one layer on n = 8192 synthetic calibration tokens, LLaMA-2-7B shape (g = 32 heads of d = 128)
+    w['llama2-7b_conversion_n8192'] = (synth.MLAShape(H=32, dn=128, dR=64, dv=128, r=512, D=4096), [8192], 9)
     for S in (128, 512, 2048, 8192):   # prefill in the MHA form: a chunk of S query positions over 8192 cached tokens
         w[f'llama2-7b-mla_prefill_b4_8k_s{S}'] = (synth.MLAShape(H=32, dn=128, dR=64, dv=128, r=512, D=4096, S=S), [8192] * 4, 8)
     return w
@@ -235,6 +237,8 @@ def run_ours(args, name, shape, seqlens, seed):
                     keep = ('config', 'ms_per_step', 'value', 'decode_kernel_us', 'cache_gbs_pct_of_8tbs', 'roofline', 'clocks')
                     if 'prefill' in row:   # a prefill row carries its own metric and the two kernels' figures
                         keep += ('metric', 'unit', 'prefill')
+                    if 'conversion_ms' in row:
+                        keep += ('metric', 'unit', 'conversion_ms')
                     line['sweep'].append({k: row[k] for k in keep})
         if world == 1 and not args.no_cpu_baseline:
             line['cpu_baseline'] = cpu_baseline(shape, seqlens, seed, (shape.dn + shape.dR) ** -0.5)
@@ -322,7 +326,97 @@ def measure_prefill(args, name, shape, seqlens, seed, rank, world, local):
     }
 
 
+def measure_conversion(args, name, shape, seqlens, seed, rank, world, local):
+    """The conversion of one layer (Sec. 4.2, 4.3; App. B, C, D) on n synthetic calibration tokens: one step = key
+    activations, per-group covariances, their eigenvectors, rotation of W_K, NoPE-key and value activations, alpha,
+    the joint second moment, the rank-r subspace (orthogonal iteration) and the rewrite of W_DKV.  fp32 SIMT
+    arithmetic: the roofline of its dominant kernel is the fp32 FMA rate."""
+    import torch
+    from paper_2502_07864_b200 import binding, replicas, synth
+    n, D, g, d, r, fold, iters = seqlens[0], shape.D, shape.H, shape.dn, shape.r, 4, 20
+    stream = torch.cuda.current_stream()
+    case = synth.make_conversion_case(n, D, g, d, seed, device='cuda')
+    x, w_k, w_v = case['x'], case['w_k'], case['w_v']
+    groups, m, mz = d // 2 // fold, g * fold, (2 * g - 1) * d
+    f32 = dict(dtype=torch.float32, device='cuda')
+    k_act, v_act, k_nope = torch.empty(n, g * d, **f32), torch.empty(n, g * d, **f32), torch.empty(n, (g - 1) * d, **f32)
+    cov, vals, U = torch.empty(groups, m, m, **f32), torch.empty(groups, m, **f32), torch.empty(groups, m, m, **f32)
+    seg = torch.empty(binding.transmla_conv_rorope_scratch_bytes(n, g, d, fold) // 4, **f32)
+    w_rot, w_dkv = torch.empty_like(w_k), torch.empty(mz, D, **f32)
+    alpha, norms = torch.zeros(1, **f32), torch.empty(2 * n, **f32)
+    Z, Cm = torch.empty(n, mz, **f32), torch.empty(mz, mz, **f32)
+    gen = torch.Generator(device='cuda'); gen.manual_seed(seed)
+    q0 = torch.randn(mz, r, generator=gen, device='cuda')
+    Q = torch.empty_like(q0)
+    ws = torch.empty(binding.transmla_conv_subspace_scratch_bytes(mz, r), dtype=torch.uint8, device='cuda')
+    out_dkv = torch.empty(r, D, **f32)
+    status = torch.zeros(1, dtype=torch.int32, device='cuda')
+    ev = {}
+
+    def mark(tag):
+        ev.setdefault(tag, []).append(torch.cuda.Event(enable_timing=True))
+        ev[tag][-1].record(stream)
+
+    def step():
+        mark('start')
+        binding.transmla_conv_gemm(x, w_k, k_act, tb=True); mark('k_act')
+        binding.transmla_conv_rorope_covariance(k_act, g, d, fold, seg, cov); mark('cov')
+        binding.transmla_conv_sym_eig(cov, vals, U, status); mark('eig')
+        binding.transmla_conv_rorope_apply(w_k, U, g, d, fold, w_rot); mark('rotate')
+        binding.transmla_conv_gemm(x, w_rot[d:], k_nope, tb=True)
+        binding.transmla_conv_gemm(x, w_v, v_act, tb=True); mark('nope_v_act')
+        binding.transmla_conv_alpha(k_nope, v_act, norms, alpha)
+        binding.transmla_conv_balance_concat(k_nope, v_act, alpha, Z); mark('alpha_concat')
+        binding.transmla_conv_gemm(Z, Z, Cm, ta=True); mark('second_moment')
+        Q.copy_(q0)
+        binding.transmla_conv_top_subspace(Cm, Q, iters, ws, status); mark('subspace')
+        w_dkv[:(g - 1) * d].copy_(w_rot[d:] / alpha); w_dkv[(g - 1) * d:].copy_(w_v)
+        binding.transmla_conv_gemm(Q, w_dkv, out_dkv, ta=True); mark('rewrite')
+
+    steps = max(2, min(args.steps, 3))
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    ev.clear()
+    sampler = ClockSampler(local) if rank == 0 else None
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step()
+    replicas.barrier('cuda')
+    t1 = time.perf_counter()
+    clocks = sampler.stop(t0, t1) if sampler else None
+    assert int(status.item()) == 0
+    tags = ['k_act', 'cov', 'eig', 'rotate', 'nope_v_act', 'alpha_concat', 'second_moment', 'subspace', 'rewrite']
+    prev = ['start'] + tags[:-1]
+    part_ms = {t: statistics.median(ev[p][i].elapsed_time(ev[t][i]) for i in range(steps)) for p, t in zip(prev, tags)}
+    ms_step = statistics.median(ev['start'][i].elapsed_time(ev['rewrite'][i]) for i in range(steps))
+    (ms_step,) = replicas.max_over_ranks([ms_step], device='cuda')
+    if rank != 0:
+        return None
+    f_sm = 2.0 * n * mz * mz
+    sm_mhz = (clocks or {}).get('sm_mhz') or 1965.0
+    peak = 148 * 128 * 2 * 1965.0e6 / 1e12     # fp32 FMA lanes x 2 flop x the maximum SM clock
+    return {
+        'metric': 'conversion of one layer: calibration tokens/s (RoRoPE + FreqFold + balanced joint PCA, synthetic activations)',
+        'value': n * world / (ms_step * 1e-3), 'unit': 'tokens/s', 'n_gpus': world, 'steps': steps, 'warmup': 3,
+        'ms_per_step': ms_step, 'higher_is_better': True, 'scaling': 'weak', 'vs_baseline': None, 'dtype': 'f32', 'data': 'synthetic',
+        'config': {'workload': name, 'calibration_tokens': n, 'hidden': D, 'kv_heads': g, 'head_dim': d, 'freqfold': fold,
+                   'rank': r, 'subspace_rounds': iters, 'l2': 'inputs larger than L2 (activations 2 x 134 MB, second moment 260 MB)',
+                   'parallelism': f'replicas x{world}, no data-path collective'},
+        'decode_kernel_us': None, 'cache_gbs_pct_of_8tbs': None,
+        'conversion_ms': part_ms,
+        'roofline': {'bound': 'alu', 'kernel': 'gemm_kernel<float> (second moment Z^T Z)', 'achieved': f_sm / part_ms['second_moment'] / 1e9,
+                     'peak': peak, 'unit': 'TFLOP/s', 'frac': f_sm / part_ms['second_moment'] / 1e9 / peak,
+                     'peak_kind': 'derived: 148 SMs x 128 fp32 lanes x 2 flop x 1965 MHz', 'traffic': None, 'flops_per_launch': f_sm,
+                     'sm_mhz_sampled': sm_mhz},
+        # gemm 6, gather 1, Jacobi 1, rotation 1, norms 3, concat 1, and (iters + 3) Cholesky QRs of three launches each
+        'gpu_launches': (13 + iters + 3 * (iters + 3)) * steps, 'clocks': clocks,
+    }
+
+
 def measure(args, name, shape, seqlens, seed, rank, world, local, full):
+    if '_conversion_' in name:
+        return measure_conversion(args, name, shape, seqlens, seed, rank, world, local)
     if '_prefill_' in name:
         return measure_prefill(args, name, shape, seqlens, seed, rank, world, local)
     """One workload: whole-step time over args.steps steps, split-KV kernel time, read-probe ceiling, and (full) the
