@@ -15,12 +15,13 @@ constexpr int BM = 128, BN = 128, BK = 8;
 template <typename TOut>
 __global__ void __launch_bounds__(256) gemm_kernel(int ta, int tb, int M, int N, int K, float alpha, const float* A, int lda,
                                                    long long strideA, const float* B, int ldb, long long strideB, TOut* C,
-                                                   int ldc, long long strideC) {
+                                                   int ldc, long long strideC, int k_total) {
   __shared__ float As[BK][BM + 4];
   __shared__ float Bs[BK][BN + 4];
   A += strideA * blockIdx.z;
   B += strideB * blockIdx.z;
   C += strideC * blockIdx.z;
+  if (k_total > 0) K = max(0, min(K, k_total - static_cast<int>(blockIdx.z) * K));  // batch = slices of one long K
   const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   TOut acc[8][8];
@@ -78,15 +79,26 @@ cudaError_t gemm_f32(int ta, int tb, int M, int N, int K, float alpha, const flo
                      cudaStream_t stream) {
   if (M <= 0 || N <= 0 || batch <= 0) return cudaSuccess;
   dim3 grid((N + BN - 1) / BN, (M + BM - 1) / BM, batch);
-  gemm_kernel<float><<<grid, 256, 0, stream>>>(ta, tb, M, N, K, alpha, A, lda, strideA, B, ldb, strideB, C, ldc, strideC);
+  gemm_kernel<float><<<grid, 256, 0, stream>>>(ta, tb, M, N, K, alpha, A, lda, strideA, B, ldb, strideB, C, ldc, strideC, 0);
   return cudaGetLastError();
 }
 
-cudaError_t gemm_f32_to_f64(int ta, int tb, int M, int N, int K, const float* A, int lda, const float* B, int ldb, double* C,
-                            int ldc, cudaStream_t stream) {
-  if (M <= 0 || N <= 0) return cudaSuccess;
-  dim3 grid((N + BN - 1) / BN, (M + BM - 1) / BM, 1);
-  gemm_kernel<double><<<grid, 256, 0, stream>>>(ta, tb, M, N, K, 1.f, A, lda, 0, B, ldb, 0, C, ldc, 0);
+// G [r,r] (fp64) = Y^T Y for Y [m,r]: the long sum over m is cut into kGramSlices slices, one batch entry each
+// (16 tiles alone would leave most SMs idle), and the partial sums are added in a fixed order.
+constexpr int kGramSlices = kGramPartials;
+__global__ void sum_slices_kernel(const double* part, int count, int slices, double* out) {
+  const int e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= count) return;
+  double s = 0.0;
+  for (int i = 0; i < slices; ++i) s += part[static_cast<size_t>(i) * count + e];
+  out[e] = s;
+}
+cudaError_t gram_f64(const float* Y, int m, int r, double* partial, double* G, cudaStream_t stream) {
+  const int ks = (m + kGramSlices - 1) / kGramSlices;
+  dim3 grid((r + BN - 1) / BN, (r + BM - 1) / BM, kGramSlices);
+  gemm_kernel<double><<<grid, 256, 0, stream>>>(1, 0, r, r, ks, 1.f, Y, r, static_cast<long long>(ks) * r, Y, r,
+                                                static_cast<long long>(ks) * r, partial, r, static_cast<long long>(r) * r, m);
+  sum_slices_kernel<<<(r * r + 255) / 256, 256, 0, stream>>>(partial, r * r, kGramSlices, G);
   return cudaGetLastError();
 }
 
@@ -322,32 +334,52 @@ cudaError_t sym_eig(float* a, int batch, int m, float* eigvals, float* eigvecs, 
 }
 // ------------------------------------------------------------------------------------------------ orthonormalisation
 // Cholesky QR: G = Y^T Y = L L^T, Q = Y L^-T.
-// cholesky_kernel: right-looking factorisation of the fp64 Gram matrix in place (one block, 32 x 32 threads over the
-// trailing block, the current column cached in shared memory); L is also written as fp32 for the solve.
-constexpr int kCholMax = 1024;
+// cholesky_kernel: blocked right-looking factorisation of the fp64 Gram matrix in place, one block.  Panels of 32
+// columns are factored in shared memory (all rows below the diagonal block with them); the trailing matrix then takes
+// one rank-32 update per panel, so that an element of G is read and written 16 times instead of 512.  L is also
+// written as fp32 for the solve.
+constexpr int kCholMax = 1024, kCholNb = 32;
 __global__ void __launch_bounds__(1024) cholesky_kernel(double* G, int r, float* L32, int32_t* dev_status) {
-  __shared__ double col[kCholMax];
+  extern __shared__ double ps[];  // panel [r - kb][kCholNb + 1]
   __shared__ int bad;
+  constexpr int ld = kCholNb + 1;
   const int tid = threadIdx.x, tx = tid & 31, ty = tid >> 5;
   if (tid == 0) bad = 0;
   __syncthreads();
-  for (int k = 0; k < r; ++k) {
-    if (tid == 0) {
-      double d = G[static_cast<size_t>(k) * r + k];
-      if (!(d > 0.0)) { bad = 1; d = 1.0; }
-      col[k] = sqrt(d);
-    }
+  for (int kb = 0; kb < r; kb += kCholNb) {
+    const int nb = min(kCholNb, r - kb), rows = r - kb;
+    for (int e = tid; e < rows * nb; e += 1024) { const int i = e / nb, j = e % nb; ps[i * ld + j] = G[static_cast<size_t>(kb + i) * r + kb + j]; }
     __syncthreads();
-    const double dk = col[k];
-    for (int i = k + 1 + tid; i < r; i += 1024) col[i] = G[static_cast<size_t>(i) * r + k] / dk;
-    __syncthreads();
-    for (int i = k + tid; i < r; i += 1024) {       // column k is final
-      G[static_cast<size_t>(i) * r + k] = col[i];
-      L32[static_cast<size_t>(i) * r + k] = static_cast<float>(col[i]);
+    for (int k = 0; k < nb; ++k) {
+      if (tid == 0) {
+        double d = ps[k * ld + k];
+        if (!(d > 0.0)) { bad = 1; d = 1.0; }
+        ps[k * ld + k] = sqrt(d);
+      }
+      __syncthreads();
+      const double dk = ps[k * ld + k];
+      for (int i = k + 1 + tid; i < rows; i += 1024) ps[i * ld + k] /= dk;
+      __syncthreads();
+      for (int e = tid; e < (rows - k - 1) * (nb - k - 1); e += 1024) {
+        const int i = k + 1 + e / (nb - k - 1), j = k + 1 + e % (nb - k - 1);
+        ps[i * ld + j] -= ps[i * ld + k] * ps[j * ld + k];
+      }
+      __syncthreads();
     }
-    for (int i = k + 1 + ty; i < r; i += 32) {      // trailing update, lower triangle only
-      const double li = col[i];
-      for (int j = k + 1 + tx; j <= i; j += 32) G[static_cast<size_t>(i) * r + j] -= li * col[j];
+    for (int e = tid; e < rows * nb; e += 1024) {
+      const int i = e / nb, j = e % nb;
+      const double v = (kb + j <= kb + i) ? ps[i * ld + j] : 0.0;
+      G[static_cast<size_t>(kb + i) * r + kb + j] = v;
+      L32[static_cast<size_t>(kb + i) * r + kb + j] = static_cast<float>(v);
+    }
+    // trailing update: G[i][j] -= sum_k P[i][k] P[j][k] for i >= j >= kb + nb
+    for (int i = nb + ty; i < rows; i += 32) {
+      for (int j = nb + tx; j <= i; j += 32) {
+        double acc = 0.0;
+#pragma unroll 8
+        for (int k = 0; k < nb; ++k) acc += ps[i * ld + k] * ps[j * ld + k];
+        G[static_cast<size_t>(kb + i) * r + kb + j] -= acc;
+      }
     }
     __syncthreads();
   }
@@ -377,10 +409,15 @@ __global__ void __launch_bounds__(256) trsm_rows_kernel(const float* Y, int m, i
   for (int c = lane; c < r; c += 32) Q[static_cast<size_t>(row) * r + c] = q[c];
 }
 
-cudaError_t cholesky_qr(const float* Y, int m, int r, double* G, float* L32, float* Q, int32_t* dev_status, cudaStream_t stream) {
+cudaError_t cholesky_qr(const float* Y, int m, int r, double* partial, double* G, float* L32, float* Q, int32_t* dev_status,
+                        cudaStream_t stream) {
   if (r > kCholMax) return cudaErrorInvalidValue;
-  if (cudaError_t e = gemm_f32_to_f64(1, 0, r, r, m, Y, r, Y, r, G, r, stream); e != cudaSuccess) return e;
-  cholesky_kernel<<<1, 1024, 0, stream>>>(G, r, L32, dev_status);
+  if (cudaError_t e = gram_f64(Y, m, r, partial, G, stream); e != cudaSuccess) return e;
+  const size_t chol_smem = static_cast<size_t>(r) * (kCholNb + 1) * sizeof(double);
+  if (cudaError_t e = cudaFuncSetAttribute(cholesky_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(chol_smem));
+      e != cudaSuccess)
+    return e;
+  cholesky_kernel<<<1, 1024, chol_smem, stream>>>(G, r, L32, dev_status);
   const size_t smem = static_cast<size_t>(8) * r * sizeof(float);
   if (smem > 48 * 1024) {
     if (cudaError_t e = cudaFuncSetAttribute(trsm_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));

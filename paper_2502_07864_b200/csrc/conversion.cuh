@@ -15,8 +15,6 @@ namespace conv {
 cudaError_t gemm_f32(int ta, int tb, int M, int N, int K, float alpha, const float* A, int lda, long long strideA,
                      const float* B, int ldb, long long strideB, float* C, int ldc, long long strideC, int batch,
                      cudaStream_t stream);
-cudaError_t gemm_f32_to_f64(int ta, int tb, int M, int N, int K, const float* A, int lda, const float* B, int ldb, double* C,
-                            int ldc, cudaStream_t stream);
 // seg[G][2n][g*fold]: rows 0..n-1 the real parts, n..2n-1 the imaginary parts of group G's dimensions (App. B, C)
 cudaError_t gather_segments(const float* K, int n, int g, int d, int fold, float* seg, cudaStream_t stream);
 // Symmetric eigendecomposition of `batch` matrices of order m <= 128 (parallel cyclic Jacobi, one block each).
@@ -28,7 +26,9 @@ cudaError_t balance_concat(const float* k_nope, int n, int mk, const float* v, i
                            cudaStream_t stream);
 // Cholesky QR: Q [m,r] = Y L^-T with Y^T Y = L L^T (Gram matrix G [r,r] and its factor in fp64; L32 [r,r] the factor
 // in fp32 for the solve).  r <= 1024.  Q may alias Y.  Sets TRANSMLA_DEV_NUMERIC if the Gram matrix is not positive definite.
-cudaError_t cholesky_qr(const float* Y, int m, int r, double* G, float* L32, float* Q, int32_t* dev_status, cudaStream_t stream);
+constexpr int kGramPartials = 8;  // partial Gram matrices [r,r] fp64 that `partial` must hold
+cudaError_t cholesky_qr(const float* Y, int m, int r, double* partial, double* G, float* L32, float* Q, int32_t* dev_status,
+                        cudaStream_t stream);
 
 }  // namespace conv
 }  // namespace transmla

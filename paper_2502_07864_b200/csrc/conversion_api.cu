@@ -69,7 +69,7 @@ transmla_status_t transmla_conv_balance_concat(const float* k_nope, int n, int m
 
 size_t transmla_conv_subspace_scratch_bytes(int m, int r) {
   if (m < 1 || r < 1 || r > m || r > 1024) return 0;
-  return static_cast<size_t>(m) * r * sizeof(float) + static_cast<size_t>(r) * r * (sizeof(double) + sizeof(float)) + 512;
+  return static_cast<size_t>(m) * r * sizeof(float) + static_cast<size_t>(r) * r * ((conv::kGramPartials + 1) * sizeof(double) + sizeof(float)) + 512;
 }
 
 transmla_status_t transmla_conv_top_subspace(const float* Cmat, int m, int r, int iters, float* Q, void* scratch,
@@ -80,12 +80,14 @@ transmla_status_t transmla_conv_top_subspace(const float* Cmat, int m, int r, in
   if (scratch_bytes < transmla_conv_subspace_scratch_bytes(m, r)) return TRANSMLA_ERR_WORKSPACE;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   char* w = static_cast<char*>(scratch);
-  double* G = reinterpret_cast<double*>(w);
+  double* partial = reinterpret_cast<double*>(w);
+  double* G = partial + static_cast<size_t>(conv::kGramPartials) * r * r;
   float* L32 = reinterpret_cast<float*>(G + static_cast<size_t>(r) * r);
-  float* Y = reinterpret_cast<float*>(w + ((static_cast<size_t>(r) * r * (sizeof(double) + sizeof(float)) + 255) & ~size_t(255)));
+  float* Y = reinterpret_cast<float*>(
+      w + ((static_cast<size_t>(r) * r * ((conv::kGramPartials + 1) * sizeof(double) + sizeof(float)) + 255) & ~size_t(255)));
   // Orthogonal iteration: Q <- orth(C Q).  One Cholesky QR per round keeps the columns independent; the basis is made
   // orthonormal to fp32 resolution by the two passes at the start and the extra pass at the end.
-  auto orth = [&](float* y, float* q) { return conv::cholesky_qr(y, m, r, G, L32, q, dev_status, s) == cudaSuccess; };
+  auto orth = [&](float* y, float* q) { return conv::cholesky_qr(y, m, r, partial, G, L32, q, dev_status, s) == cudaSuccess; };
   if (!orth(Q, Q) || !orth(Q, Q)) return TRANSMLA_ERR_CUDA;
   for (int it = 0; it < iters; ++it) {
     if (conv::gemm_f32(0, 0, m, r, m, 1.f, Cmat, m, 0, Q, r, 0, Y, r, 0, 1, s) != cudaSuccess) return TRANSMLA_ERR_CUDA;
