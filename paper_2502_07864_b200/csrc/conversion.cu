@@ -8,57 +8,106 @@ namespace transmla {
 namespace conv {
 
 // ------------------------------------------------------------------------------------------------ GEMM
-// 128 x 128 tile, 256 threads x (8 x 8) outputs, k in steps of 8 through shared memory.  Any of the four
-// storage combinations; edges are bounds-checked, so no shape restriction.
-constexpr int BM = 128, BN = 128, BK = 8;
+// 128 x 128 tile, 256 threads x (8 x 8) outputs, k in steps of 16 through two shared-memory buffers: the next
+// tile's global loads (16 bytes each where the storage allows, element by element at ragged edges or odd strides)
+// are in flight while the current tile is multiplied.  Any of the four storage combinations, no shape restriction.
+constexpr int BM = 128, BN = 128, BK = 16;
+
+// One operand tile [128 x BK] as two float4 per thread.  `rows_major`: the operand is stored [rows, K] (k contiguous),
+// otherwise [K, rows] (rows contiguous).  r0 = first row of the tile, R = row count, ld = storage stride.
+struct TileRegs { float4 v[2]; };
+__device__ __forceinline__ void fetch_tile(TileRegs& t, const float* P, bool rows_major, bool vec, int ld, int r0, int R, int k0,
+                                           int K, int tid) {
+#pragma unroll
+  for (int u = 0; u < 2; ++u) {
+    const int f = tid + 256 * u;
+    float x[4] = {0.f, 0.f, 0.f, 0.f};
+    if (rows_major) {
+      const int rr = r0 + f / 4, k = k0 + (f % 4) * 4;
+      if (rr < R) {
+        const float* src = P + static_cast<size_t>(rr) * ld + k;
+        if (vec && k + 3 < K) { const float4 q = *reinterpret_cast<const float4*>(src); x[0] = q.x; x[1] = q.y; x[2] = q.z; x[3] = q.w; }
+        else {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) if (k + c < K) x[c] = src[c];
+        }
+      }
+    } else {
+      const int k = k0 + f / 32, rr = r0 + (f % 32) * 4;
+      if (k < K) {
+        const float* src = P + static_cast<size_t>(k) * ld + rr;
+        if (vec && rr + 3 < R) { const float4 q = *reinterpret_cast<const float4*>(src); x[0] = q.x; x[1] = q.y; x[2] = q.z; x[3] = q.w; }
+        else {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) if (rr + c < R) x[c] = src[c];
+        }
+      }
+    }
+    t.v[u] = make_float4(x[0], x[1], x[2], x[3]);
+  }
+}
+__device__ __forceinline__ void stash_tile(const TileRegs& t, float (*S)[BM + 4], bool rows_major, int tid) {
+#pragma unroll
+  for (int u = 0; u < 2; ++u) {
+    const int f = tid + 256 * u;
+    if (rows_major) {
+      const int rr = f / 4, kq = (f % 4) * 4;
+      S[kq][rr] = t.v[u].x; S[kq + 1][rr] = t.v[u].y; S[kq + 2][rr] = t.v[u].z; S[kq + 3][rr] = t.v[u].w;
+    } else {
+      *reinterpret_cast<float4*>(&S[f / 32][(f % 32) * 4]) = t.v[u];
+    }
+  }
+}
 
 template <typename TOut>
 __global__ void __launch_bounds__(256) gemm_kernel(int ta, int tb, int M, int N, int K, float alpha, const float* A, int lda,
                                                    long long strideA, const float* B, int ldb, long long strideB, TOut* C,
                                                    int ldc, long long strideC, int k_total) {
-  __shared__ float As[BK][BM + 4];
-  __shared__ float Bs[BK][BN + 4];
+  __shared__ __align__(16) float As[2][BK][BM + 4];
+  __shared__ __align__(16) float Bs[2][BK][BN + 4];
   A += strideA * blockIdx.z;
   B += strideB * blockIdx.z;
   C += strideC * blockIdx.z;
   if (k_total > 0) K = max(0, min(K, k_total - static_cast<int>(blockIdx.z) * K));  // batch = slices of one long K
   const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const bool a_rows = !ta, b_rows = tb != 0;   // stored [rows, K]?
+  const bool vec_a = (lda & 3) == 0 && (reinterpret_cast<uintptr_t>(A) & 15) == 0;
+  const bool vec_b = (ldb & 3) == 0 && (reinterpret_cast<uintptr_t>(B) & 15) == 0;
   TOut acc[8][8];
 #pragma unroll
   for (int i = 0; i < 8; ++i)
 #pragma unroll
     for (int j = 0; j < 8; ++j) acc[i][j] = TOut(0);
+  TileRegs ra, rb;
+  if (K > 0) {
+    fetch_tile(ra, A, a_rows, vec_a, lda, m0, M, 0, K, tid);
+    fetch_tile(rb, B, b_rows, vec_b, ldb, n0, N, 0, K, tid);
+    stash_tile(ra, As[0], a_rows, tid);
+    stash_tile(rb, Bs[0], b_rows, tid);
+  }
+  __syncthreads();
   for (int k0 = 0; k0 < K; k0 += BK) {
-    // tile loads: walk the contiguous storage dimension with consecutive threads
-    for (int e = tid; e < BM * BK; e += 256) {
-      int mm, kk;
-      if (ta) { mm = e % BM; kk = e / BM; } else { kk = e % BK; mm = e / BK; }
-      const int m = m0 + mm, k = k0 + kk;
-      float v = 0.f;
-      if (m < M && k < K) v = ta ? A[static_cast<size_t>(k) * lda + m] : A[static_cast<size_t>(m) * lda + k];
-      As[kk][mm] = v;
+    const int buf = (k0 / BK) & 1;
+    const bool more = k0 + BK < K;
+    if (more) {
+      fetch_tile(ra, A, a_rows, vec_a, lda, m0, M, k0 + BK, K, tid);
+      fetch_tile(rb, B, b_rows, vec_b, ldb, n0, N, k0 + BK, K, tid);
     }
-    for (int e = tid; e < BN * BK; e += 256) {
-      int nn, kk;
-      if (tb) { kk = e % BK; nn = e / BK; } else { nn = e % BN; kk = e / BN; }
-      const int n = n0 + nn, k = k0 + kk;
-      float v = 0.f;
-      if (n < N && k < K) v = tb ? B[static_cast<size_t>(n) * ldb + k] : B[static_cast<size_t>(k) * ldb + n];
-      Bs[kk][nn] = v;
-    }
-    __syncthreads();
 #pragma unroll
     for (int kk = 0; kk < BK; ++kk) {
-      float a[8], b[8];
-#pragma unroll
-      for (int i = 0; i < 8; ++i) a[i] = As[kk][ty * 4 + (i & 3) + (i >> 2) * 64];
-#pragma unroll
-      for (int j = 0; j < 8; ++j) b[j] = Bs[kk][tx * 4 + (j & 3) + (j >> 2) * 64];
+      const float4 a0 = *reinterpret_cast<const float4*>(&As[buf][kk][ty * 4]), a1 = *reinterpret_cast<const float4*>(&As[buf][kk][64 + ty * 4]);
+      const float4 b0 = *reinterpret_cast<const float4*>(&Bs[buf][kk][tx * 4]), b1 = *reinterpret_cast<const float4*>(&Bs[buf][kk][64 + tx * 4]);
+      const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+      const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
 #pragma unroll
       for (int i = 0; i < 8; ++i)
 #pragma unroll
         for (int j = 0; j < 8; ++j) acc[i][j] += static_cast<TOut>(a[i]) * static_cast<TOut>(b[j]);
+    }
+    if (more) {
+      stash_tile(ra, As[buf ^ 1], a_rows, tid);
+      stash_tile(rb, Bs[buf ^ 1], b_rows, tid);
     }
     __syncthreads();
   }
