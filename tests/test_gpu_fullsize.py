@@ -153,3 +153,30 @@ def test_full_size_closed_forms_cover_every_output(shape, B):
         want = w_uv @ c
         for s in range(shape.S):
             gu.assert_close(got[b, s], want, f'identical rows b={b} s={s}')
+
+
+def test_prefill_chunk_of_2048_positions_over_8192_tokens_sampled():
+    # the prefill workload bench.py times (B = 4 x 8192 cached tokens, S = 2048): sampled (sequence, position, head)
+    # outputs against the oracle, among them the first and last position of the chunk and both sides of a 128-row tile
+    shape = synth.MLAShape(H=32, dn=128, dR=64, dv=128, r=512, D=4096, S=2048)
+    seqlens = [8192] * 4
+    scale = gu.mla_scale(shape)
+    case = synth.make_decode_case(shape, seqlens, 8, device='cuda')
+    params = binding.make_params(shape, 4, case['cache'].shape[0], case['page_table'].shape[1], scale)
+    scratch = torch.empty(binding.transmla_prefill_scratch_bytes(params) // 2, dtype=torch.bfloat16, device='cuda')
+    status = torch.zeros(1, dtype=torch.int32, device='cuda')
+    out = torch.full((4, 2048, 32, 128), float('nan'), dtype=torch.bfloat16, device='cuda')
+    lse = torch.full((4, 2048, 32), float('nan'), dtype=torch.float32, device='cuda')
+    binding.transmla_mla_prefill(params, case['q_nope'], case['q_pe'], case['w_uk'], case['w_uv'], case['cache'],
+                                 case['page_table'], case['seqlens'], scratch, out, lse, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and torch.all(torch.isfinite(out.float()))
+    seqs = [0, 3]
+    sub = sub_case(case, seqs)
+    rng = np.random.default_rng(8)
+    positions = [0, 1, 127, 128, 1000, 2047]
+    only = [(i, s, int(h)) for i in range(len(seqs)) for s in positions for h in rng.choice(32, size=2, replace=False)]
+    want, want_lse = gu.oracle_decode(shape, sub, scale, only=only)
+    idx = tuple(np.array(only).T)
+    gu.assert_close(lifts.f64(out[seqs])[idx], want[idx], 'prefill sampled outputs at the benchmark size')
+    gu.assert_lse_close(lifts.f64(lse[seqs])[idx], want_lse[idx], 'prefill sampled lse')
