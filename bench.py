@@ -42,6 +42,8 @@ def workloads():
     w['llama2-7b_conversion_n8192'] = (synth.MLAShape(H=32, dn=128, dR=64, dv=128, r=512, D=4096), [8192], 9)
     for S in (128, 512, 2048, 8192):   # prefill in the MHA form: a chunk of S query positions over 8192 cached tokens
         w[f'llama2-7b-mla_prefill_b4_8k_s{S}'] = (synth.MLAShape(H=32, dn=128, dR=64, dv=128, r=512, D=4096, S=S), [8192] * 4, 8)
+        if S <= 2048:   # the headline batch; 2.6 GB of decompressed keys and values
+            w[f'llama2-7b-mla_prefill_b16_8k_s{S}'] = (synth.MLAShape(H=32, dn=128, dR=64, dv=128, r=512, D=4096, S=S), [8192] * 16, 8)
     return w
 
 
@@ -646,7 +648,7 @@ def main():
     ap.add_argument('--q-lora-rank', type=int, default=0, help='low-rank queries for --layer (0: full rank)')
     ap.add_argument('--layer-weight-copies', type=int, default=6)
     ap.add_argument('--sweep', default='llama2-7b-mla_b64_8k,llama2-7b-mla_b128_8k,qwen2.5-72b-mla_b64_s2,llama2-7b-mla-fp8_b64_8k,'
-                            'llama2-7b-mla_prefill_b4_8k_s2048',
+                            'llama2-7b-mla_prefill_b16_8k_s2048',
                     help='comma-separated workloads measured after the main one (1 GPU; empty: none)')
     args = ap.parse_args()
     w = workloads()

@@ -107,7 +107,8 @@ def lib():
         for name in EXPORTS:
             if name not in ('transmla_step_staging_bytes', 'transmla_status_string',
                             'transmla_profile_decode_kernel', 'transmla_static_workspace_capacity',
-                            'transmla_layer_scratch_bytes'):
+                            'transmla_layer_scratch_bytes', 'transmla_prefill_scratch_bytes',
+                            'transmla_conv_rorope_scratch_bytes', 'transmla_conv_subspace_scratch_bytes'):
                 getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib

@@ -39,6 +39,17 @@ def test_workspace_layout_is_host_arithmetic():
         assert off % 256 == 0
 
 
+def test_byte_counts_beyond_4_gib_come_back_whole():
+    # host arithmetic only; the counts are size_t and must not pass through a 32-bit return type
+    build.build()
+    shape = synth.MLAShape(H=32, dn=128, dR=64, dv=128, r=512, D=4096, S=16)
+    params = binding.make_params(shape, 16, 4096, 128, 0.07)
+    assert binding.transmla_prefill_scratch_bytes(params) == 4096 * 64 * 32 * 256 * 2
+    assert binding.transmla_conv_rorope_scratch_bytes(1 << 20, 32, 128, 4) == 16 * 2 * (1 << 20) * 128 * 4
+    assert binding.transmla_conv_subspace_scratch_bytes(100000, 1024) > (1 << 28)
+    assert binding.transmla_prefill_scratch_bytes(binding.make_params(synth.TINY, 2, 4, 2, 0.1)) == 0
+
+
 def test_shape_errors_are_codes():
     s = synth.LLAMA2_7B
     lay = binding.WorkspaceLayout()
