@@ -306,6 +306,43 @@ def test_decode_step_from_host_buffers(pinned):
     gu.assert_lse_close(lifts.f64(h_lse), want_lse, 'host step lse')
 
 
+def test_host_step_repeated_with_new_contents_in_the_same_buffers():
+    # three consecutive steps through the same pinned buffers, staging and workspace: every call must read the
+    # buffers' current contents (new queries, a new token, sequences one token longer)
+    shape = synth.LLAMA2_7B
+    B = 2
+    scale = gu.mla_scale(shape)
+    dc = synth.make_decode_case(shape, [300, 129], 25, extra_pages=2)
+    params = binding.make_params(shape, B, dc['cache'].shape[0], dc['page_table'].shape[1], scale)
+    ws, _ = binding.alloc_workspace(params)
+    staging = torch.empty(binding.transmla_step_staging_bytes(params), dtype=torch.uint8, device='cuda')
+    pin = lambda t: t.contiguous().pin_memory()
+    h = {k: pin(dc[k]) for k in ('q_nope', 'q_pe', 'page_table', 'seqlens')}
+    h_x = pin(torch.empty(B, 1, shape.D, dtype=torch.bfloat16))
+    h_out = pin(torch.empty(B, 1, shape.H, shape.dv, dtype=torch.bfloat16))
+    cache = dc['cache'].cuda()
+    want_cache = lifts.f64(dc['cache'])
+    w = synth.make_append_case(shape, [0, 0], 26)['w_dkv_kr']
+    w_dev, w_uk, w_uv = w.cuda(), dc['w_uk'].cuda(), dc['w_uv'].cuda()
+    seqlens = [300, 129]
+    for it in range(3):
+        ac = synth.make_append_case(shape, [L - 1 for L in seqlens], 30 + it)
+        qn = synth.make_decode_case(shape, seqlens, 40 + it)
+        h_x.copy_(ac['x']); h['q_nope'].copy_(qn['q_nope']); h['q_pe'].copy_(qn['q_pe'])
+        h['seqlens'].copy_(torch.tensor(seqlens, dtype=torch.int32))
+        word = binding.transmla_decode_step_host(params, h_x, h['q_nope'], h['q_pe'], h['page_table'], h['seqlens'], w_dev,
+                                                 w_uk, w_uv, cache, staging, ws, h_out)
+        assert word == 0
+        orc.latent_append(lifts.f64(ac['x'][:, 0]), lifts.f64(w), [L - 1 for L in seqlens], dc['page_table'].numpy(),
+                          want_cache, shape.r)
+        want_cache = lifts.f64(torch.tensor(want_cache).to(torch.bfloat16))
+        case = dict(dc, q_nope=qn['q_nope'], q_pe=qn['q_pe'], cache=torch.tensor(want_cache).to(torch.bfloat16),
+                    seqlens=torch.tensor(seqlens, dtype=torch.int32))
+        want, _ = gu.oracle_decode(shape, case, scale)
+        gu.assert_close(lifts.f64(h_out), want, f'repeated host step {it}')
+        seqlens = [L + 1 for L in seqlens]
+
+
 # ------------------------------------------------------------------ whole layer: queries, attention, W_O
 @pytest.mark.parametrize('shape,seqlens,rq', [(synth.TINY, [17, 64, 130], 0), (synth.TINY, [5, 70], 256),
                                                (synth.LLAMA2_7B, [300, 65, 1024], 0), (synth.LLAMA2_7B, [200, 64], 512),
